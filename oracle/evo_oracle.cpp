@@ -1,0 +1,349 @@
+// Reference oracle for the candidate-evaluation step (TEST INFRASTRUCTURE ONLY).
+//
+// A plain, slow, single-threaded CPU statement of what the evaluation step of
+// the EvoEngineer method computes: seeded trial inputs, the functional-
+// correctness constraint g(p) (paper Section 3.1, Eq. 1; Section 4.3 "Modular
+// Architecture Design", functional testing: outputs are compared against the
+// reference implementation over the test cases) and the runtime objective f(p)
+// (Section 4.3: times collected over repeated runs; Section 5.1 "Evaluation
+// Metric": speedup over the baseline kernel).
+//
+// This file is used by the tests, by the smoke check and by the benchmark's CPU
+// baseline leg only.  It shares no code, header, table or constant generator
+// with the CUDA library and the product never calls it.
+//
+// Build: g++ -std=c++17 -O2 -ffp-contract=off -fno-fast-math (see build.py).
+// Contraction must stay off: the closeness rule is defined on individually
+// rounded binary32 operations.
+//
+// Pins (tests/test_oracle_*.py): Philox known-answer vectors; Box-Muller against
+// 50-digit evaluation, distribution tests and closed-form invariants; narrowing
+// against numpy/torch conversions; the closeness rule against a table of
+// hand-worked cases, torch.isclose, an exhaustive 16-bit sweep evaluated through
+// double, and brute force; medians against the statistics module.
+// No function here is "parity unpinned".
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <vector>
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy
+// as 1, 2, 3", SC'11).  The paper only says that the test inputs are random
+// (Section 4.3: five test cases; Appendix A.8.1 "Evaluation Method": five
+// random inputs); the generator is fixed by this library's interface.
+// ---------------------------------------------------------------------------
+constexpr uint32_t kMul0 = 0xD2511F53u;  // multiplier applied to counter word 0
+constexpr uint32_t kMul1 = 0xCD9E8D57u;  // multiplier applied to counter word 2
+constexpr uint32_t kWeyl0 = 0x9E3779B9u; // key word 0 increment per round
+constexpr uint32_t kWeyl1 = 0xBB67AE85u; // key word 1 increment per round
+
+void philox_round(uint32_t c[4], const uint32_t k[2]) {
+    const uint64_t p0 = static_cast<uint64_t>(kMul0) * c[0];
+    const uint64_t p1 = static_cast<uint64_t>(kMul1) * c[2];
+    const uint32_t hi0 = static_cast<uint32_t>(p0 >> 32), lo0 = static_cast<uint32_t>(p0);
+    const uint32_t hi1 = static_cast<uint32_t>(p1 >> 32), lo1 = static_cast<uint32_t>(p1);
+    const uint32_t n0 = hi1 ^ c[1] ^ k[0];
+    const uint32_t n1 = lo1;
+    const uint32_t n2 = hi0 ^ c[3] ^ k[1];
+    const uint32_t n3 = lo0;
+    c[0] = n0; c[1] = n1; c[2] = n2; c[3] = n3;
+}
+
+void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    uint32_t c[4] = {ctr[0], ctr[1], ctr[2], ctr[3]};
+    uint32_t k[2] = {key[0], key[1]};
+    for (int round = 0; round < 10; ++round) {
+        if (round > 0) { k[0] += kWeyl0; k[1] += kWeyl1; }
+        philox_round(c, k);
+    }
+    for (int i = 0; i < 4; ++i) out[i] = c[i];
+}
+
+// Stream layout: element g of the stream of `seed` is word (g mod 4) of the
+// Philox block whose counter is (lo32(g/4), hi32(g/4), 0, 0) under the key
+// (lo32(seed), hi32(seed)).
+uint32_t stream_word(uint64_t seed, uint64_t g) {
+    const uint64_t b = g >> 2;
+    const uint32_t ctr[4] = {static_cast<uint32_t>(b), static_cast<uint32_t>(b >> 32), 0u, 0u};
+    const uint32_t key[2] = {static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32)};
+    uint32_t out[4];
+    philox4x32_10(ctr, key, out);
+    return out[g & 3];
+}
+
+// ---------------------------------------------------------------------------
+// Box-Muller.  Words pair up inside a block: (x0,x1) -> (z0,z1), (x2,x3) ->
+// (z2,z3).  u1 = ((xa >> 8) + 1) / 2^24 in (0, 1];  u2 = (xb >> 8) / 2^24 in
+// [0, 1).  z_even = sqrt(-2 ln u1) cos(2 pi u2), z_odd = sqrt(-2 ln u1)
+// sin(2 pi u2).  Evaluated in double; the angle is reduced by quadrant on the
+// integer so that the exact zeros of sin/cos at multiples of pi/2 stay exact.
+// ---------------------------------------------------------------------------
+void box_muller(uint32_t xa, uint32_t xb, double* z_cos, double* z_sin) {
+    const double u1 = (static_cast<double>(xa >> 8) + 1.0) / 16777216.0;
+    const uint32_t k = xb >> 8;                 // angle = 2 pi k / 2^24
+    const uint32_t quadrant = k >> 22;          // 0..3
+    const uint32_t m = k & ((1u << 22) - 1u);   // position inside the quadrant
+    const double half_pi = 1.57079632679489661923132169163975144;
+    // Inside the quadrant measure the angle from the nearer axis, so that the
+    // value next to a zero crossing keeps full relative accuracy.
+    double s, c;
+    if (m <= (1u << 21)) {
+        const double phi = half_pi * (static_cast<double>(m) / 4194304.0);
+        s = std::sin(phi); c = std::cos(phi);
+    } else {
+        const double psi = half_pi * (static_cast<double>((1u << 22) - m) / 4194304.0);
+        s = std::cos(psi); c = std::sin(psi);
+    }
+    double cosv, sinv;
+    switch (quadrant) {
+        case 0: cosv = c;  sinv = s;  break;
+        case 1: cosv = -s; sinv = c;  break;
+        case 2: cosv = -c; sinv = -s; break;
+        default: cosv = s; sinv = -c; break;
+    }
+    const double rho = std::sqrt(-2.0 * std::log(u1));
+    *z_cos = rho * cosv;
+    *z_sin = rho * sinv;
+}
+
+double normal_f64(uint64_t seed, uint64_t g) {
+    const uint64_t pair_first = g & ~static_cast<uint64_t>(1);
+    const uint32_t xa = stream_word(seed, pair_first);
+    const uint32_t xb = stream_word(seed, pair_first + 1);
+    double zc, zs;
+    box_muller(xa, xb, &zc, &zs);
+    return (g & 1) ? zs : zc;
+}
+
+// ---------------------------------------------------------------------------
+// Storage formats.  Widening is exact; narrowing is round-to-nearest-even.
+// ---------------------------------------------------------------------------
+uint32_t f32_bits(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
+float bits_f32(uint32_t u) { float f; std::memcpy(&f, &u, 4); return f; }
+
+float widen_bf16(uint16_t h) { return bits_f32(static_cast<uint32_t>(h) << 16); }
+
+float widen_f16(uint16_t h) {
+    const uint32_t sign = (h & 0x8000u) ? 0x80000000u : 0u;
+    const int e = (h >> 10) & 0x1f;
+    const uint32_t frac = h & 0x3ffu;
+    if (e == 0x1f) return bits_f32(sign | 0x7f800000u | (frac << 13));       // Inf / NaN
+    if (e == 0) {                                                             // zero / subnormal
+        const float mag = std::ldexp(static_cast<float>(frac), -24);          // exact
+        return sign ? -mag : mag;
+    }
+    return bits_f32(sign | (static_cast<uint32_t>(e - 15 + 127) << 23) | (frac << 13));
+}
+
+uint16_t narrow_bf16(float f) {
+    const uint32_t u = f32_bits(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return static_cast<uint16_t>((u >> 16) | 0x0040u);  // NaN stays NaN
+    const uint32_t lower = u & 0xffffu;
+    uint32_t upper = u >> 16;
+    if (lower > 0x8000u || (lower == 0x8000u && (upper & 1u))) upper += 1;   // carry into exponent is correct
+    return static_cast<uint16_t>(upper);
+}
+
+uint16_t narrow_f16(float f) {
+    const uint32_t u = f32_bits(f);
+    const uint16_t sign = static_cast<uint16_t>((u >> 16) & 0x8000u);
+    const uint32_t absu = u & 0x7fffffffu;
+    if (absu > 0x7f800000u) return static_cast<uint16_t>(sign | 0x7e00u);     // NaN
+    if (absu == 0x7f800000u) return static_cast<uint16_t>(sign | 0x7c00u);    // Inf
+    const double mag = std::fabs(static_cast<double>(f));
+    if (mag == 0.0) return sign;
+    // Scale so that one unit is the spacing of the target format at this
+    // magnitude, round to nearest even on the integer, rebuild.
+    int e;
+    std::frexp(mag, &e);                       // mag = m * 2^e, m in [0.5, 1)
+    int exp_unbiased = e - 1;                  // mag in [2^exp, 2^(exp+1))
+    if (exp_unbiased < -14) exp_unbiased = -14;  // subnormal spacing is fixed at 2^-24
+    const double spacing = std::ldexp(1.0, exp_unbiased - 10);
+    const double scaled = mag / spacing;       // exact (power-of-two scaling)
+    double r = std::floor(scaled);
+    const double rem = scaled - r;
+    if (rem > 0.5 || (rem == 0.5 && std::fmod(r, 2.0) == 1.0)) r += 1.0;
+    const double rounded = r * spacing;
+    if (rounded >= 65520.0) return static_cast<uint16_t>(sign | 0x7c00u);     // overflows to Inf
+    if (rounded < std::ldexp(1.0, -14)) {                                     // subnormal or zero
+        return static_cast<uint16_t>(sign | static_cast<uint16_t>(rounded / std::ldexp(1.0, -24)));
+    }
+    int e2;
+    const double m2 = std::frexp(rounded, &e2);   // rounded = m2 * 2^e2, m2 in [0.5,1)
+    const int biased = (e2 - 1) + 15;
+    const uint32_t frac = static_cast<uint32_t>((m2 * 2.0 - 1.0) * 1024.0);
+    return static_cast<uint16_t>(sign | (static_cast<uint32_t>(biased) << 10) | frac);
+}
+
+enum { DT_U32 = 0, DT_F32 = 1, DT_F16 = 2, DT_BF16 = 3 };
+
+float load_widened(const void* p, uint64_t i, int dtype) {
+    switch (dtype) {
+        case DT_F32:  return static_cast<const float*>(p)[i];
+        case DT_F16:  return widen_f16(static_cast<const uint16_t*>(p)[i]);
+        default:      return widen_bf16(static_cast<const uint16_t*>(p)[i]);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+struct oracle_result {
+    uint64_t n_mismatch;
+    uint64_t n_nonfinite;
+    double sse;
+    float max_abs;
+    float max_rel;
+    uint32_t flags;   // 1 cand NaN, 2 cand +Inf, 4 cand -Inf, 8 ref NaN, 16 ref +-Inf
+    uint32_t pass;
+};
+
+struct oracle_fit {
+    float median_ms;
+    float speedup;
+    uint32_t valid;
+    uint32_t status;  // 0 ok, 1 a candidate time is not finite and positive, 2 same for a baseline time
+};
+
+void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
+    philox4x32_10(ctr, key, out);
+}
+
+// The transform alone: two words -> (z_even, z_odd), unrounded.
+void oracle_box_muller(uint32_t xa, uint32_t xb, double* out2) { box_muller(xa, xb, &out2[0], &out2[1]); }
+
+void oracle_gen_u32(uint64_t seed, uint64_t offset, uint64_t n, uint32_t* out) {
+    for (uint64_t i = 0; i < n; ++i) out[i] = stream_word(seed, offset + i);
+}
+
+// Unrounded (double) normals, for ulp measurements.
+void oracle_gen_normal_f64(uint64_t seed, uint64_t offset, uint64_t n, double* out) {
+    for (uint64_t i = 0; i < n; ++i) out[i] = normal_f64(seed, offset + i);
+}
+
+// dtype 0: raw words; 1: fp32 normals (one rounding from double); 2/3: the
+// fp32 value narrowed once more to fp16 / bf16.
+int oracle_gen_inputs(uint64_t seed, uint64_t offset, int dtype, uint64_t n, void* out) {
+    if (dtype == DT_U32) { oracle_gen_u32(seed, offset, n, static_cast<uint32_t*>(out)); return 0; }
+    if (dtype != DT_F32 && dtype != DT_F16 && dtype != DT_BF16) return -3;
+    for (uint64_t i = 0; i < n; ++i) {
+        const float z = static_cast<float>(normal_f64(seed, offset + i));
+        if (dtype == DT_F32) static_cast<float*>(out)[i] = z;
+        else if (dtype == DT_F16) static_cast<uint16_t*>(out)[i] = narrow_f16(z);
+        else static_cast<uint16_t*>(out)[i] = narrow_bf16(z);
+    }
+    return 0;
+}
+
+void oracle_narrow(int dtype, const float* in, uint64_t n, uint16_t* out) {
+    for (uint64_t i = 0; i < n; ++i) out[i] = (dtype == DT_F16) ? narrow_f16(in[i]) : narrow_bf16(in[i]);
+}
+
+void oracle_widen(int dtype, const uint16_t* in, uint64_t n, float* out) {
+    for (uint64_t i = 0; i < n; ++i) out[i] = (dtype == DT_F16) ? widen_f16(in[i]) : widen_bf16(in[i]);
+}
+
+// Closeness rule for one element, every operation a single binary32 rounding:
+//   d = |c - r|;  tol = atol + rtol * |r|;  close = (c == r) or (d finite and d <= tol).
+// Returns 1 when the element is a mismatch.
+int oracle_element_mismatch(float c, float r, float atol, float rtol) {
+    const float diff = c - r;
+    const float d = std::fabs(diff);
+    const float t = rtol * std::fabs(r);
+    const float tol = atol + t;
+    const bool close = (c == r) || (std::isfinite(d) && d <= tol);
+    return close ? 0 : 1;
+}
+
+// The correctness constraint over one tensor (Section 3.1 Eq. 1, g(p); Section
+// 4.3 functional testing), plus the error statistics reported with it.
+// Elements where c or r is NaN/Inf are counted and flagged, judged by the rule
+// above, and left out of max_abs, max_rel and sse.  max_rel skips r == 0.
+int oracle_validate(const void* cand, const void* ref, uint64_t n, int dtype,
+                    float atol, float rtol, oracle_result* out) {
+    if (dtype != DT_F32 && dtype != DT_F16 && dtype != DT_BF16) return -3;
+    oracle_result res{};
+    res.max_abs = 0.0f;
+    res.max_rel = 0.0f;
+    double sse = 0.0;
+    for (uint64_t i = 0; i < n; ++i) {
+        const float c = load_widened(cand, i, dtype);
+        const float r = load_widened(ref, i, dtype);
+        res.n_mismatch += static_cast<uint64_t>(oracle_element_mismatch(c, r, atol, rtol));
+        bool nonfinite = false;
+        if (std::isnan(c)) { res.flags |= 1u; nonfinite = true; }
+        if (std::isinf(c)) { res.flags |= (c > 0.0f) ? 2u : 4u; nonfinite = true; }
+        if (std::isnan(r)) { res.flags |= 8u; nonfinite = true; }
+        if (std::isinf(r)) { res.flags |= 16u; nonfinite = true; }
+        if (nonfinite) { res.n_nonfinite += 1; continue; }
+        const float d = std::fabs(c - r);
+        if (d > res.max_abs) res.max_abs = d;
+        if (r != 0.0f) {
+            const float q = d / std::fabs(r);
+            if (q > res.max_rel) res.max_rel = q;
+        }
+        sse += static_cast<double>(d) * static_cast<double>(d);
+    }
+    res.sse = sse;
+    res.pass = (res.n_mismatch == 0) ? 1u : 0u;
+    *out = res;
+    return 0;
+}
+
+// A candidate is valid when every one of its output tensors / test cases
+// passes: AND over the descriptors carrying the same group id.
+void oracle_group_pass(const oracle_result* results, const uint32_t* group, uint64_t n_desc,
+                       uint32_t* group_pass, uint64_t n_group) {
+    for (uint64_t g = 0; g < n_group; ++g) group_pass[g] = 1u;
+    for (uint64_t i = 0; i < n_desc; ++i)
+        if (group[i] < n_group && !results[i].pass) group_pass[group[i]] = 0u;
+}
+
+// Median of a row of run times: the middle order statistic, or the mean of the
+// two middle ones (each operation one binary32 rounding).  Returns false when a
+// time is not finite and positive.
+static bool row_median(const float* row, uint32_t trials, float* median) {
+    std::vector<float> v(row, row + trials);
+    for (float x : v) if (!(std::isfinite(x) && x > 0.0f)) return false;
+    std::sort(v.begin(), v.end());
+    if (trials & 1u) { *median = v[trials / 2]; return true; }
+    const float s = v[trials / 2 - 1] + v[trials / 2];
+    *median = 0.5f * s;
+    return true;
+}
+
+// Objective f(p): speedup of the candidate over the baseline kernel from the
+// medians of their run times (Section 4.3 timing protocol; Appendix A.7.1
+// "Limitations and Threats to Validity" states that the median of the runs is
+// taken; Section 5.1 "Evaluation Metric": speedup over the baseline).  A
+// candidate that failed the constraint gets valid = 0 and speedup 0.
+int oracle_fitness(const float* times, uint64_t n_cand, uint32_t trials,
+                   const float* base_times, uint32_t base_trials,
+                   const uint32_t* pass, oracle_fit* out) {
+    if (trials == 0 || base_trials == 0) return -1;
+    float base_median = 0.0f;
+    const bool base_ok = row_median(base_times, base_trials, &base_median);
+    for (uint64_t i = 0; i < n_cand; ++i) {
+        oracle_fit f{};
+        float med = 0.0f;
+        const bool ok = row_median(times + i * static_cast<uint64_t>(trials), trials, &med);
+        if (!ok) { f.status = 1u; }
+        else if (!base_ok) { f.status = 2u; f.median_ms = med; }
+        else {
+            f.median_ms = med;
+            const bool passed = (pass == nullptr) || (pass[i] != 0u);
+            if (passed) { f.valid = 1u; f.speedup = base_median / med; }
+        }
+        out[i] = f;
+    }
+    return 0;
+}
+
+}  // extern "C"

@@ -1,0 +1,162 @@
+"""ctypes front end of the CPU oracle (oracle/evo_oracle.cpp).
+
+Test infrastructure only.  Every function takes and returns numpy arrays on the
+host; nothing here touches CUDA or imports the product package.
+"""
+import ctypes as C
+
+import numpy as np
+
+from . import build as _build
+
+U32, F32, F16, BF16 = 0, 1, 2, 3
+_ELEM_BYTES = {U32: 4, F32: 4, F16: 2, BF16: 2}
+
+RESULT_DTYPE = np.dtype(
+    [("n_mismatch", "<u8"), ("n_nonfinite", "<u8"), ("sse", "<f8"), ("max_abs", "<f4"),
+     ("max_rel", "<f4"), ("flags", "<u4"), ("pass", "<u4")], align=True)
+FIT_DTYPE = np.dtype(
+    [("median_ms", "<f4"), ("speedup", "<f4"), ("valid", "<u4"), ("status", "<u4")], align=True)
+assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(_build.build())
+        L.oracle_philox4x32_10.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_philox4x32_10.restype = None
+        L.oracle_box_muller.argtypes = [C.c_uint32, C.c_uint32, C.c_void_p]
+        L.oracle_box_muller.restype = None
+        L.oracle_gen_u32.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p]
+        L.oracle_gen_u32.restype = None
+        L.oracle_gen_normal_f64.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64, C.c_void_p]
+        L.oracle_gen_normal_f64.restype = None
+        L.oracle_gen_inputs.argtypes = [C.c_uint64, C.c_uint64, C.c_int, C.c_uint64, C.c_void_p]
+        L.oracle_gen_inputs.restype = C.c_int
+        L.oracle_narrow.argtypes = [C.c_int, C.c_void_p, C.c_uint64, C.c_void_p]
+        L.oracle_narrow.restype = None
+        L.oracle_widen.argtypes = [C.c_int, C.c_void_p, C.c_uint64, C.c_void_p]
+        L.oracle_widen.restype = None
+        L.oracle_element_mismatch.argtypes = [C.c_float, C.c_float, C.c_float, C.c_float]
+        L.oracle_element_mismatch.restype = C.c_int
+        L.oracle_validate.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_int, C.c_float, C.c_float, C.c_void_p]
+        L.oracle_validate.restype = C.c_int
+        L.oracle_group_pass.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64]
+        L.oracle_group_pass.restype = None
+        L.oracle_fitness.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
+        L.oracle_fitness.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _ptr(a):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def philox4x32_10(counter, key):
+    """One Philox4x32-10 block: counter (4 x u32), key (2 x u32) -> 4 x u32."""
+    c = np.ascontiguousarray(counter, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    assert c.shape == (4,) and k.shape == (2,)
+    out = np.empty(4, dtype=np.uint32)
+    lib().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def box_muller(xa, xb):
+    """Two stream words -> (z_even, z_odd) in double, before rounding."""
+    out = np.empty(2, dtype=np.float64)
+    lib().oracle_box_muller(int(xa) & 0xFFFFFFFF, int(xb) & 0xFFFFFFFF, _ptr(out))
+    return float(out[0]), float(out[1])
+
+
+def gen_u32(seed, offset, n):
+    out = np.empty(int(n), dtype=np.uint32)
+    lib().oracle_gen_u32(int(seed), int(offset), int(n), _ptr(out))
+    return out
+
+
+def gen_normal_f64(seed, offset, n):
+    """Standard normals of the stream before any rounding to a storage type."""
+    out = np.empty(int(n), dtype=np.float64)
+    lib().oracle_gen_normal_f64(int(seed), int(offset), int(n), _ptr(out))
+    return out
+
+
+def gen_inputs(seed, offset, dtype, n):
+    """Raw words (U32 -> uint32), fp32 normals (F32 -> float32) or the bit
+    patterns of fp16/bf16 normals (F16/BF16 -> uint16)."""
+    np_dt = {U32: np.uint32, F32: np.float32, F16: np.uint16, BF16: np.uint16}[dtype]
+    out = np.empty(int(n), dtype=np_dt)
+    rc = lib().oracle_gen_inputs(int(seed), int(offset), int(dtype), int(n), _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_gen_inputs: status %d" % rc)
+    return out
+
+
+def narrow(dtype, x):
+    """fp32 -> fp16/bf16 bit patterns, round-to-nearest-even."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint16)
+    lib().oracle_narrow(int(dtype), _ptr(x), x.size, _ptr(out))
+    return out
+
+
+def widen(dtype, bits):
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(bits.shape, dtype=np.float32)
+    lib().oracle_widen(int(dtype), _ptr(bits), bits.size, _ptr(out))
+    return out
+
+
+def element_mismatch(c, r, atol, rtol):
+    return int(lib().oracle_element_mismatch(float(np.float32(c)), float(np.float32(r)),
+                                             float(np.float32(atol)), float(np.float32(rtol))))
+
+
+def validate(cand, ref, dtype, atol, rtol):
+    """One candidate tensor against its reference.  `cand`/`ref` are float32
+    arrays (F32) or uint16 bit patterns (F16/BF16).  Returns a RESULT_DTYPE scalar."""
+    np_dt = np.float32 if dtype == F32 else np.uint16
+    cand = np.ascontiguousarray(cand)
+    ref = np.ascontiguousarray(ref)
+    if cand.dtype != np_dt or ref.dtype != np_dt:
+        raise TypeError("validate: arrays must be %s for dtype %d" % (np_dt, dtype))
+    if cand.size != ref.size:
+        raise ValueError("validate: size mismatch")
+    out = np.zeros(1, dtype=RESULT_DTYPE)
+    rc = lib().oracle_validate(_ptr(cand), _ptr(ref), cand.size, int(dtype),
+                               float(np.float32(atol)), float(np.float32(rtol)), _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_validate: status %d" % rc)
+    return out[0]
+
+
+def group_pass(results, group, n_group):
+    results = np.ascontiguousarray(results, dtype=RESULT_DTYPE)
+    group = np.ascontiguousarray(group, dtype=np.uint32)
+    out = np.empty(int(n_group), dtype=np.uint32)
+    lib().oracle_group_pass(_ptr(results), _ptr(group), results.size, _ptr(out), int(n_group))
+    return out
+
+
+def fitness(times, base_times, passed=None):
+    """times [n_cand, trials] fp32, base_times [base_trials] fp32, passed optional
+    [n_cand] u32.  Returns a FIT_DTYPE array of n_cand entries."""
+    times = np.ascontiguousarray(times, dtype=np.float32)
+    base = np.ascontiguousarray(base_times, dtype=np.float32)
+    assert times.ndim == 2 and base.ndim == 1
+    n_cand, trials = times.shape
+    p = None
+    if passed is not None:
+        p = np.ascontiguousarray(passed, dtype=np.uint32)
+        assert p.shape == (n_cand,)
+    out = np.zeros(n_cand, dtype=FIT_DTYPE)
+    rc = lib().oracle_fitness(_ptr(times), n_cand, trials, _ptr(base), base.size,
+                              _ptr(p) if p is not None else None, _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_fitness: status %d" % rc)
+    return out
