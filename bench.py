@@ -1,0 +1,392 @@
+#!/usr/bin/env python
+"""Benchmark of the candidate-evaluation step on B200.
+
+One "step" is one pass of the whole evaluation path over one population of synthetic
+candidate outputs: evo_gen_inputs (one test-input tensor), evo_validate (every candidate
+tensor against its reference) and evo_fitness (median-of-trials speedup).  The metric is the
+rate at which candidate outputs are validated: algorithmic bytes (every candidate tensor once,
+every distinct reference once) per second, for inputs already resident in HBM (`value`) and
+through the host-buffer entry points with the copies inside the timed region (`e2e`).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4|config3|config5|config2]
+    python bench.py --impl reference ...     # the CPU oracle on a bounded sample (baseline arm)
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank evaluates its own
+replica of the population: candidates are independent, there is no exchange between GPUs.
+"""
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads  # noqa: E402
+
+METRIC = "validated_bytes_per_second"
+UNIT = "GB/s"
+WORKLOAD_NOTES = {
+    "config4": "16 fp32 candidates x 2^28 elements (1 GiB each) sharing one 1 GiB reference",
+    "config3": "64 fp16 + 64 bf16 candidates x 2^20 elements, one reference per dtype",
+    "config5": "1024 candidates, 1-3 tensors each, 2^10..2^24 elements, fp32/fp16/bf16, own references",
+    "config2": "8 fp32 candidates x 262144 elements sharing one reference (fits in L2)",
+}
+
+
+def build_population(name, device):
+    return getattr(workloads, name)(device)
+
+
+def gen_elems(pop):
+    """Size of the test-input tensor generated per step: one tensor as large as the largest output."""
+    return max(t.cand.numel() for t in pop.tensors)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while a region runs."""
+
+    def __init__(self, index, period_s=0.02):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ----------------------------------------------------------------------------- oracle arm
+FULL_SHAPE = {"config4": dict(n=1 << 28, k=16), "config3": dict(n=1 << 20, k=128), "config2": dict(n=1 << 18, k=8)}
+
+
+class OracleSample:
+    """A bounded sample of a workload for the CPU oracle, and the factors that scale its
+    timings (linear in elements) to one full step of that workload."""
+
+    def __init__(self, workload, log2_elems, log2_gen):
+        if workload in FULL_SHAPE:
+            n_full, k_full = FULL_SHAPE[workload]["n"], FULL_SHAPE[workload]["k"]
+            n_s = min(n_full, 1 << log2_elems)
+            if workload == "config4":
+                pop = workloads.config4("cpu", n=n_s, k=4)
+            elif workload == "config3":
+                pop = workloads.config3("cpu", n=n_s, k_per_dtype=2)
+            else:
+                pop = workloads.config2("cpu", n=n_s, k=4)
+            self.scale_val = (n_full * k_full) / float(n_s * len(pop.tensors))
+            self.rows, self.n_gen_full = k_full, n_full
+            what = "%d candidates x 2^%d elements of %s" % (len(pop.tensors), n_s.bit_length() - 1, workload)
+        else:
+            pop = workloads.config5("cpu", n_cand=48, log2_min=10.0, log2_max=float(min(22, log2_elems)))
+            self.scale_val = 2048 * 1.73e6 / float(sum(t.cand.numel() for t in pop.tensors))
+            self.rows, self.n_gen_full = 1024, 1 << 24
+            what = "48 candidates of config5 with sizes up to 2^%d" % min(22, log2_elems)
+        self.pop = pop
+        self.refs = [workloads.to_host_bits(r) for r in pop.refs]
+        self.cands = [workloads.to_host_bits(t.cand) for t in pop.tensors]
+        self.n_gen = min(self.n_gen_full, 1 << log2_gen)
+        import numpy as np
+        self.times = np.repeat(pop.times.numpy()[:1], self.rows, axis=0)
+        self.base = pop.base_times.numpy()
+        self.description = ("oracle, 1 thread: validate %s, generate 2^%d normals, fitness of %d rows; "
+                            "timings scaled linearly in elements to one full step" % (what, self.n_gen.bit_length() - 1, self.rows))
+
+    def run(self):
+        """One timed pass over the sample; returns (estimated seconds of a full step, seconds spent)."""
+        import oracle
+        t0 = time.perf_counter()
+        for t, c in zip(self.pop.tensors, self.cands):
+            oracle.validate(c, self.refs[t.ref_index], t.dtype, self.pop.atol, self.pop.rtol)
+        t1 = time.perf_counter()
+        oracle.gen_inputs(1, 0, oracle.F32, self.n_gen)
+        t2 = time.perf_counter()
+        oracle.fitness(self.times, self.base)
+        t3 = time.perf_counter()
+        est = (t1 - t0) * self.scale_val + (t2 - t1) * (self.n_gen_full / float(self.n_gen)) + (t3 - t2)
+        return est, t3 - t0
+
+
+def full_algorithmic_bytes(workload):
+    known = {"config4": 17 * (1 << 30), "config3": 130 * (1 << 21), "config2": 9 * (1 << 20)}
+    return known.get(workload, int(2048 * 1.73e6 * 3 * 2))
+
+
+def run_reference(args):
+    """Baseline arm: the CPU oracle, as it stands, on the host cores; rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    passes = args.steps + args.warmup
+    log2 = 24 if passes <= 30 else 22 if passes <= 120 else 20 if passes <= 500 else 18   # about 1 s .. 20 ms per pass
+    sample = OracleSample(args.workload, log2, log2 - 2)
+    alg_bytes = full_algorithmic_bytes(args.workload)
+    for _ in range(args.warmup):
+        sample.run()
+    ests, spent = [], 0.0
+    for _ in range(args.steps):
+        est, s = sample.run()
+        ests.append(est)
+        spent += s
+    est = sum(ests) / len(ests)
+    value = alg_bytes / est / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "what": WORKLOAD_NOTES[args.workload],
+                   "note": "ms_per_step is the time of one full step estimated from the timed sample"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.description},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "sample_seconds_per_step": spent / max(1, args.steps),
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- GPU arm
+def run_ours(args):
+    import paper_2510_03760_b200 as evo
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    distributed = world > 1
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if distributed:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if distributed:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ctx = evo.Context(local_rank)
+    pop = build_population(args.workload, device)
+    cands = [t.cand for t in pop.tensors]
+    refs = [pop.refs[t.ref_index] for t in pop.tensors]
+    groups = [t.group for t in pop.tensors]
+    n_group = pop.n_group
+    alg_bytes = pop.algorithmic_bytes()
+    n_gen = gen_elems(pop)
+    gen_buf = torch.empty(n_gen, dtype=torch.float32, device=device)
+    results = torch.empty((len(cands), 40), dtype=torch.uint8, device=device)
+    gpass = torch.empty(n_group, dtype=torch.int32, device=device)
+    fits = torch.empty((n_group, 16), dtype=torch.uint8, device=device)
+
+    def step(i, ev=None):
+        evo.evo_gen_inputs(1000 + i, 0, evo.EVO_F32, n_gen, gen_buf, ctx=ctx)
+        if ev is not None:
+            ctx.set_timing_events(ev[0], ev[1])
+        evo.evo_validate(cands, refs, pop.atol, pop.rtol, groups=groups, n_group=n_group, results=results,
+                         group_pass=gpass, ctx=ctx)
+        evo.evo_fitness(pop.times, pop.base_times, gpass, out=fits, ctx=ctx)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    barrier()
+
+    # per-step event pairs around the main validation kernel (recorded once so the handles exist)
+    kern_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in kern_events:
+        a.record()
+        b.record()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(torch.cuda._get_nvml_device_index(local_rank) if hasattr(torch.cuda, "_get_nvml_device_index") else local_rank)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches_before = ctx.launches
+    with sampler:
+        barrier()
+        start.record()
+        for i in range(args.steps):
+            step(i, kern_events[i])
+        stop.record()
+        barrier()
+    launches = ctx.launches - launches_before
+    total_ms = start.elapsed_time(stop)
+    kern_ms = [a.elapsed_time(b) for a, b in kern_events]
+    if distributed:
+        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * alg_bytes / (ms_per_step * 1e-3) / 1e9
+    cand_per_s = world * n_group / (ms_per_step * 1e-3)
+
+    # correctness spot check of the timed configuration: verdicts known by construction
+    res = evo.results_to_numpy(results)
+    if "wrong" in pop.facts:
+        assert res["pass"].sum() == len(cands) - 1 and res["pass"][pop.facts["wrong"]] == 0, "verdicts are wrong"
+
+    # ---- end to end through the host-buffer entry points (pinned host tensors) ----
+    e2e = None
+    if not args.no_e2e:
+        import psutil
+        need = alg_bytes + (2 << 30)
+        if psutil.virtual_memory().available > 2 * need and torch.cuda.mem_get_info()[0] > need:
+            h_refs = [r.cpu().pin_memory() for r in pop.refs]
+            h_cands = [t.cand.cpu().pin_memory() for t in pop.tensors]
+            aliasing = False
+        else:  # not enough host memory for a second copy of the population: reuse two host tensors
+            h_refs = [r.cpu().pin_memory() for r in pop.refs[:1]]
+            one = pop.tensors[0].cand.cpu().pin_memory()
+            h_cands = [one for _ in pop.tensors]
+            aliasing = True
+        h_refl = [h_refs[t.ref_index if not aliasing else 0] for t in pop.tensors]
+        h_times, h_base = pop.times.cpu().numpy(), pop.base_times.cpu().numpy()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+
+        def e2e_step(i):
+            evo.evo_gen_inputs(2000 + i, 0, evo.EVO_F32, n_gen, gen_buf, ctx=ctx)
+            r, gp = evo.evo_validate_host(h_cands, h_refl, pop.atol, pop.rtol, groups=groups, n_group=n_group,
+                                          device=local_rank, ctx=ctx)
+            f = evo.evo_fitness_host(h_times, h_base, gp, device=local_rank, ctx=ctx)
+            return r, gp, f
+
+        e2e_step(0)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            r, gp, f = e2e_step(i)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if distributed:
+            t = torch.tensor([dt], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        h2d = alg_bytes + h_times.nbytes + h_base.nbytes + gp.nbytes
+        d2h = r.nbytes + gp.nbytes + f.nbytes
+        e2e = {"value": world * alg_bytes / (dt / e2e_steps) / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "steps": e2e_steps, "ms_per_step": dt / e2e_steps * 1e3,
+               "host_memory": "pinned", "timer": "host wall clock around synchronous calls, max over ranks",
+               "host_tensors_aliased": aliasing}
+        del h_cands, h_refs, h_refl
+
+    if rank != 0:
+        if distributed:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    kern_avg_ms = sum(kern_ms) / len(kern_ms)
+    achieved = alg_bytes / (kern_avg_ms * 1e-3) / 1e9
+    traffic = None   # set from an ncu capture of this kernel version, see profiles/
+    tpath = os.path.join(ROOT, "profiles", "validate_pass1_traffic.json")
+    if os.path.exists(tpath):
+        try:
+            tj = json.load(open(tpath))
+            if tj.get("workload") == args.workload:
+                traffic = tj.get("dram_bytes_per_launch")
+        except Exception:
+            traffic = None
+    roofline = {"kernel": "validate_pass1", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": UNIT,
+                "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": traffic,
+                "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms_avg": kern_avg_ms,
+                "kernel_ms_min": min(kern_ms), "kernel_ms_max": max(kern_ms)}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        sample = OracleSample(args.workload, 27, 25)          # about 10-20 s of single-thread work
+        est, spent = sample.run()
+        cpu = {"value": alg_bytes / est / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.description,
+               "seconds": spent, "host_cores_available": os.cpu_count()}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "what": WORKLOAD_NOTES[args.workload],
+                   "step": "evo_gen_inputs(%d fp32 normals) + evo_validate(%d tensors) + evo_fitness(%d x %d trials)"
+                           % (n_gen, len(cands), n_group, pop.times.shape[1]),
+                   "algorithmic_bytes_per_step": alg_bytes, "l2": "inputs larger than L2" if alg_bytes > (1 << 28) else "inputs fit in L2",
+                   "replicas": world},
+        "candidates_per_s": cand_per_s, "frac_of_hbm_peak": value / world / peak,
+        "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": roofline, "cpu_baseline": cpu,
+    }
+    print(json.dumps(line))
+    if distributed:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=sorted(WORKLOAD_NOTES), default="config4")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,238 @@
+/*
+ * evo.h - C ABI of the candidate-evaluation library (CUDA, sm_100a).
+ *
+ * The EvoEngineer paper states kernel optimisation as a constrained problem
+ * (Section 3.1, Eq. 1): minimise a performance objective f(p) subject to a
+ * correctness constraint g(p) = 0, and reports validity rate and median speedup
+ * as metrics (Section 5.1 "Evaluation Metric").  Its evaluator (Section 4.3
+ * "Modular Architecture Design") runs functional testing on random test inputs
+ * against the reference implementation and then times the kernel over repeated
+ * runs.  This library is the data-parallel part of that evaluator:
+ *
+ *   evo_gen_inputs   seeded random test inputs            (Section 4.3; Appendix A.8.1 "Evaluation Method")
+ *   evo_validate     the functional-correctness part of g (Section 3.1 Eq. 1; Section 4.3 functional testing)
+ *   evo_fitness      f: median run time -> speedup         (Section 4.3 timing; Appendix A.7.1; Section 5.1)
+ *
+ * The paper fixes neither the random generator, nor the comparison formula, nor
+ * the treatment of NaN/Inf; those are fixed here and stated with each call.
+ *
+ * Conventions
+ *   - Every function returns an int status: EVO_OK (0) or a negative EVO_ERR_*.
+ *     Nothing throws, aborts or traps.  evo_last_error() gives a message for the
+ *     last failing call on a context.
+ *   - "device" pointers are CUDA device addresses on the context's device; "host"
+ *     pointers are ordinary process memory.  The caller owns every buffer it
+ *     passes; the library keeps no pointer to them after the call's stream work
+ *     has run.
+ *   - Calls taking a `stream` (a cudaStream_t passed as void*, NULL = the default
+ *     stream) only enqueue work; results are in device memory once the stream
+ *     reaches that point.  The *_host variants synchronise the stream before they
+ *     return.
+ *   - A context owns a scratch workspace that grows on demand (cudaMalloc inside
+ *     the call that needs it, never during stream capture by design of the
+ *     caller) and is released by evo_destroy.  Use one context per stream; calls
+ *     on one context must not overlap on the device.
+ *   - There is no CPU fallback: without a CUDA device every call but
+ *     evo_strerror fails with EVO_ERR_CUDA.
+ */
+#ifndef EVO_H_
+#define EVO_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define EVO_API __attribute__((visibility("default")))
+#else
+#define EVO_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    EVO_OK = 0,
+    EVO_ERR_ARG = -1,        /* null pointer, bad count, tolerance negative or not finite, ... */
+    EVO_ERR_ALIGN = -2,      /* pointer not aligned to its element size */
+    EVO_ERR_DTYPE = -3,      /* dtype code not accepted by this call */
+    EVO_ERR_CUDA = -4,       /* a CUDA runtime call failed; evo_last_error has its text */
+    EVO_ERR_WORKSPACE = -5,  /* scratch memory could not be obtained or a fixed limit was exceeded */
+    EVO_ERR_TIMEOUT = -6     /* a bounded device-side wait gave up (reported through the context status word) */
+};
+
+/* Element types. EVO_U32 is accepted by evo_gen_inputs only. */
+enum { EVO_U32 = 0, EVO_F32 = 1, EVO_F16 = 2, EVO_BF16 = 3 };
+
+/* Bits of evo_result.flags. */
+enum {
+    EVO_FLAG_CAND_NAN = 1, EVO_FLAG_CAND_PINF = 2, EVO_FLAG_CAND_NINF = 4,
+    EVO_FLAG_REF_NAN = 8, EVO_FLAG_REF_INF = 16
+};
+
+typedef struct evo_ctx evo_ctx;
+
+/* Create / destroy a context bound to CUDA device `device`.  evo_create allocates
+ * a small workspace; evo_destroy synchronises the device work of the context's
+ * last calls and frees everything the context owns. */
+EVO_API int evo_create(evo_ctx** ctx, int device);
+EVO_API int evo_destroy(evo_ctx* ctx);
+
+/* Static text for a status code; never NULL. */
+EVO_API const char* evo_strerror(int status);
+/* Message of the last failing call on `ctx` (owned by the context, valid until
+ * the next call on it); "" if none. */
+EVO_API const char* evo_last_error(const evo_ctx* ctx);
+
+/*
+ * evo_gen_inputs - fill `out` with n elements of the random stream of `seed`,
+ * starting at stream position `offset` (counted in elements, any value).
+ * Paper: test inputs are random (Section 4.3, five test cases; Appendix A.8.1,
+ * five random inputs).  Generator (fixed here): Philox4x32-10 (Salmon et al.,
+ * SC'11).  Stream element g is word (g mod 4) of the block with counter
+ * (lo32(g/4), hi32(g/4), 0, 0) under key (lo32(seed), hi32(seed)), so
+ * gen(seed, a, n)[i] == gen(seed, 0, a + n)[a + i] for every a.
+ *   dtype EVO_U32 : the raw words.
+ *   dtype EVO_F32 : standard normals by Box-Muller on word pairs (x0,x1),(x2,x3) of a block:
+ *                   u1 = ((xa >> 8) + 1) / 2^24,  u2 = (xb >> 8) / 2^24,
+ *                   z_even = sqrt(-2 ln u1) cos(2 pi u2),  z_odd = sqrt(-2 ln u1) sin(2 pi u2),
+ *                   computed in binary32 (within 4 ulp of the exactly rounded value).
+ *   dtype EVO_F16 / EVO_BF16 : the binary32 value rounded to nearest even.
+ * out: device, n elements of the type, aligned to the element size, written
+ * completely.  n == 0 is a no-op.  Errors: EVO_ERR_ARG (null ctx/out),
+ * EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_CUDA.
+ */
+EVO_API int evo_gen_inputs(evo_ctx* ctx, uint64_t seed, uint64_t offset, int dtype, uint64_t n,
+                   void* out /* device */, void* stream);
+
+/* One candidate output tensor to check. */
+typedef struct {
+    uint64_t n;        /* elements; 0 is legal (passes, all statistics zero) */
+    const void* ref;   /* device; NULL = use the call's ref_ptr */
+    int32_t dtype;     /* EVO_F32/F16/BF16; -1 = use the call's dtype.  Candidate and reference share it. */
+    uint32_t group;    /* candidate id in [0, n_group): tensors / test cases of one candidate share a verdict */
+} evo_desc;
+
+typedef struct {
+    uint64_t n_mismatch;   /* elements violating the closeness rule */
+    uint64_t n_nonfinite;  /* elements where candidate or reference is NaN or +-Inf */
+    double sse;            /* sum of d^2 over elements with both values finite */
+    float max_abs;         /* max d over those elements (0 if none; +Inf if a finite difference overflows) */
+    float max_rel;         /* max d / |r| over those elements with r != 0 (0 if none) */
+    uint32_t flags;        /* EVO_FLAG_* */
+    uint32_t pass;         /* 1 iff n_mismatch == 0 */
+} evo_result;              /* 40 bytes */
+
+/*
+ * evo_validate - the functional-correctness constraint over a population.
+ * Paper: Section 3.1 Eq. 1 (g(p) = 0, "output must match the reference
+ * implementation across test cases"); Section 4.3 (functional testing against
+ * the reference outputs).  Rule (fixed here), per element, candidate c and
+ * reference r widened exactly to binary32, each operation rounded once, no fused
+ * multiply-add, subnormals kept:
+ *     d = |c - r|,  tol = atol + rtol * |r|,
+ *     close = (c == r) or (d is finite and d <= tol);   mismatch = not close.
+ * So NaN never matches, equal infinities match (but are flagged), +0 matches -0.
+ * Elements with a NaN/Inf on either side are counted in n_nonfinite, flagged,
+ * judged by the rule, and left out of max_abs, max_rel and sse.
+ *
+ * cand_ptrs : host array of n_desc device pointers, one candidate tensor each.
+ * ref_ptr   : device reference shared by all descriptors whose .ref is NULL (may be NULL if none is).
+ * descs     : host array of n_desc descriptors.  Descriptors with the same (reference, n, dtype)
+ *             are found and their reference is read from memory once for all of them.
+ * dtype     : default element type for descriptors with .dtype == -1.
+ * atol,rtol : finite and >= 0.
+ * results   : device, n_desc entries, written completely; entry i belongs to descriptor i.
+ * group_pass: device, n_group words, optional (NULL with n_group 0): word g = AND of .pass over the
+ *             descriptors with .group == g (1 for a group without descriptors).
+ * Tensors need only element alignment; 16-byte aligned tensors take the fast path.
+ * The host arrays are consumed before the call returns.  n_desc == 0 is legal.
+ * Errors: EVO_ERR_ARG, EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_WORKSPACE, EVO_ERR_CUDA.
+ */
+EVO_API int evo_validate(evo_ctx* ctx, const void* const* cand_ptrs /* host array of device ptrs */,
+                 const void* ref_ptr /* device */, const evo_desc* descs /* host */, uint64_t n_desc,
+                 int dtype, float atol, float rtol, evo_result* results /* device */,
+                 uint32_t* group_pass /* device, optional */, uint64_t n_group, void* stream);
+
+/*
+ * evo_validate_host - the same check for tensors that live in host memory: every
+ * pointer (cand_ptrs[i], ref_ptr, descs[i].ref, results, group_pass) is a HOST
+ * address.  The tensors are copied to a staging area owned by the context
+ * (distinct references once), checked there by the same kernels, and the results
+ * are copied back; the stream is synchronised before returning.  Pinned host
+ * memory makes the copies faster but is not required.
+ */
+EVO_API int evo_validate_host(evo_ctx* ctx, const void* const* cand_ptrs /* host array of host ptrs */,
+                      const void* ref_ptr /* host */, const evo_desc* descs /* host */, uint64_t n_desc,
+                      int dtype, float atol, float rtol, evo_result* results /* host */,
+                      uint32_t* group_pass /* host, optional */, uint64_t n_group, void* stream);
+
+typedef struct {
+    float median_ms;   /* median of the candidate's run times (0 if status == 1) */
+    float speedup;     /* baseline median / candidate median; 0 if not valid */
+    uint32_t valid;    /* 1 iff status == 0 and the candidate passed (pass NULL = all passed) */
+    uint32_t status;   /* 0 ok; 1 a candidate time is NaN, Inf or <= 0; 2 a baseline time is */
+} evo_fit;             /* 16 bytes */
+
+/*
+ * evo_fitness - the performance objective f(p): speedup over the baseline kernel
+ * from the medians of the run times.
+ * Paper: Section 4.3 (run times collected over 100 runs); Appendix A.7.1 (the
+ * median of multiple runs is taken; Section 4.3 says "average": the two passages
+ * disagree, the median is what this call computes); Section 5.1 "Evaluation
+ * Metric" (speedup over the baseline).  Median = middle order statistic, or
+ * 0.5 * (a + b) of the two middle ones; speedup = base_median / median; all in
+ * binary32, one rounding per operation.  The floor of 1.0 that the paper applies
+ * when reporting across kernels is not applied here.
+ * times      : device, n_cand rows of `trials` floats (milliseconds), row-major.
+ * base_times : device, base_trials floats.
+ * pass       : device, n_cand words (e.g. group_pass of evo_validate), optional.
+ * out        : device, n_cand entries.
+ * 1 <= trials, base_trials <= 4096.  Errors: EVO_ERR_ARG, EVO_ERR_CUDA.
+ */
+EVO_API int evo_fitness(evo_ctx* ctx, const float* times /* device */, uint64_t n_cand, uint32_t trials,
+                const float* base_times /* device */, uint32_t base_trials,
+                const uint32_t* pass /* device, optional */, evo_fit* out /* device */, void* stream);
+
+/* evo_fitness for host arrays (all four pointers are HOST addresses); synchronises the stream. */
+EVO_API int evo_fitness_host(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials,
+                     const float* base_times, uint32_t base_trials,
+                     const uint32_t* pass, evo_fit* out, void* stream);
+
+/*
+ * evo_plan_inspect - host-only view of the schedule evo_validate would use on a device that
+ * runs `max_ctas` persistent CTAs: how descriptors were merged into sets that share one
+ * reference read, and which contiguous run of (set, tile) items each CTA walks.  Touches no
+ * device and dereferences no tensor; meant for inspection and for testing the scheduler.
+ * (The persistent grid over ragged descriptors is this library's design; the paper has no
+ * counterpart.)
+ * summary    : host, written.
+ * ranges     : host, optional, max_ctas entries; entry b is CTA b's run
+ *              [(set_begin, tile_begin), (set_end, tile_end)), tile_end exclusive inside
+ *              set_end; set_begin > set_end marks an idle CTA.
+ * set_of_desc: host, optional, n_desc entries: the set each descriptor joined.
+ * set_k      : host, optional, n_desc entries (only the first n_sets are written): members per set.
+ * Errors: as evo_validate's argument checks.
+ */
+typedef struct { uint32_t n_sets, n_ctas, n_parts, tile_bytes; uint64_t total_tiles; } evo_plan_summary;
+typedef struct { uint64_t tile_begin, tile_end; uint32_t set_begin, set_end; } evo_plan_range;
+EVO_API int evo_plan_inspect(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs, uint64_t n_desc,
+                             int dtype, uint32_t max_ctas, evo_plan_summary* summary, evo_plan_range* ranges,
+                             uint32_t* set_of_desc, uint32_t* set_k);
+
+/*
+ * evo_set_timing_events - ask the next evo_validate / evo_validate_host call on `ctx` to record
+ * two CUDA events (cudaEvent_t passed as void*, created by the caller with timing enabled) on
+ * its stream: `start` right before and `stop` right after the launch of the main checking
+ * kernel (the first pass over the tensors).  The request is consumed by that call; pass NULLs
+ * to cancel.  For measuring the kernel alone inside a longer stream of work.  (The paper has
+ * no counterpart.)
+ */
+EVO_API int evo_set_timing_events(evo_ctx* ctx, void* start, void* stop);
+
+/* Number of kernels this context has launched so far (for accounting in benchmarks). */
+EVO_API uint64_t evo_launch_count(const evo_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EVO_H_ */

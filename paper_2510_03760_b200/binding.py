@@ -1,0 +1,247 @@
+"""ctypes binding of libevo (include/evo.h).  Argument marshalling only: every step of the
+evaluation runs in the library's kernels.  torch supplies device memory and streams."""
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+EVO_U32, EVO_F32, EVO_F16, EVO_BF16 = 0, 1, 2, 3
+_TORCH_TO_CODE = {torch.float32: EVO_F32, torch.float16: EVO_F16, torch.bfloat16: EVO_BF16}
+
+RESULT_DTYPE = np.dtype(
+    [("n_mismatch", "<u8"), ("n_nonfinite", "<u8"), ("sse", "<f8"), ("max_abs", "<f4"),
+     ("max_rel", "<f4"), ("flags", "<u4"), ("pass", "<u4")], align=True)
+FIT_DTYPE = np.dtype(
+    [("median_ms", "<f4"), ("speedup", "<f4"), ("valid", "<u4"), ("status", "<u4")], align=True)
+_DESC_DTYPE = np.dtype([("n", "<u8"), ("ref", "<u8"), ("dtype", "<i4"), ("group", "<u4")], align=True)
+assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16 and _DESC_DTYPE.itemsize == 24
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libevo.so")
+_lib = None
+
+
+class EvoError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__("libevo status %d: %s" % (status, message))
+        self.status = status
+
+
+def load_library():
+    """Load libevo.so.  Fails loudly if it has not been built: there is no other code path."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError("%s is missing: build it with `python -m paper_2510_03760_b200.build`" % _LIB_PATH)
+    L = C.CDLL(_LIB_PATH)
+    vp, u64, u32, i32, f32 = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int, C.c_float
+    L.evo_create.argtypes = [C.POINTER(vp), i32]
+    L.evo_create.restype = i32
+    L.evo_destroy.argtypes = [vp]
+    L.evo_destroy.restype = i32
+    L.evo_strerror.argtypes = [i32]
+    L.evo_strerror.restype = C.c_char_p
+    L.evo_last_error.argtypes = [vp]
+    L.evo_last_error.restype = C.c_char_p
+    L.evo_launch_count.argtypes = [vp]
+    L.evo_launch_count.restype = u64
+    L.evo_set_timing_events.argtypes = [vp, vp, vp]
+    L.evo_set_timing_events.restype = i32
+    L.evo_gen_inputs.argtypes = [vp, u64, u64, i32, u64, vp, vp]
+    L.evo_gen_inputs.restype = i32
+    for name in ("evo_validate", "evo_validate_host"):
+        fn = getattr(L, name)
+        fn.argtypes = [vp, vp, vp, vp, u64, i32, f32, f32, vp, vp, u64, vp]
+        fn.restype = i32
+    for name in ("evo_fitness", "evo_fitness_host"):
+        fn = getattr(L, name)
+        fn.argtypes = [vp, vp, u64, u32, vp, u32, vp, vp, vp]
+        fn.restype = i32
+    _lib = L
+    return L
+
+
+class Context:
+    """Owns an evo_ctx (device workspace).  One per stream in use."""
+
+    def __init__(self, device=0):
+        L = load_library()
+        h = C.c_void_p()
+        st = L.evo_create(C.byref(h), int(device))
+        if st != 0:
+            raise EvoError(st, L.evo_strerror(st).decode())
+        self._h = h
+        self.device = int(device)
+
+    def check(self, status):
+        if status != 0:
+            L = load_library()
+            raise EvoError(status, "%s (%s)" % (L.evo_strerror(status).decode(), L.evo_last_error(self._h).decode()))
+
+    @property
+    def launches(self):
+        return int(load_library().evo_launch_count(self._h))
+
+    def set_timing_events(self, start, stop):
+        """Have the next evo_validate on this context record torch CUDA events (created with
+        enable_timing=True and already recorded once, so that their handles exist) around its
+        main kernel."""
+        st = load_library().evo_set_timing_events(
+            self._h, C.c_void_p(start.cuda_event) if start is not None else None,
+            C.c_void_p(stop.cuda_event) if stop is not None else None)
+        self.check(st)
+
+    def close(self):
+        if self._h is not None and _lib is not None:
+            _lib.evo_destroy(self._h)
+        self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+_default_ctx = {}
+
+
+def default_context(device=None):
+    device = torch.cuda.current_device() if device is None else int(device)
+    ctx = _default_ctx.get(device)
+    if ctx is None:
+        ctx = _default_ctx[device] = Context(device)
+    return ctx
+
+
+def dtype_code(t):
+    try:
+        return _TORCH_TO_CODE[t]
+    except KeyError:
+        raise TypeError("unsupported tensor dtype %s" % t)
+
+
+def _stream_ptr(stream, device):
+    if stream is None:
+        stream = torch.cuda.current_stream(device)
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _dev_ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def evo_gen_inputs(seed, offset, dtype, n, out, stream=None, ctx=None):
+    """Fill the first n elements of the CUDA tensor `out` (uint32/int32 storage for EVO_U32,
+    float32/float16/bfloat16 otherwise) with the stream of `seed` from position `offset`."""
+    if not out.is_cuda or not out.is_contiguous() or out.numel() < n:
+        raise ValueError("out must be a contiguous CUDA tensor with at least n elements")
+    want = {EVO_U32: 4, EVO_F32: 4, EVO_F16: 2, EVO_BF16: 2}.get(dtype)
+    if want is not None and out.element_size() != want:
+        raise ValueError("out has the wrong element size for dtype %d" % dtype)
+    ctx = ctx or default_context(out.device.index)
+    st = load_library().evo_gen_inputs(ctx._h, int(seed), int(offset), int(dtype), int(n), _dev_ptr(out),
+                                       _stream_ptr(stream, out.device))
+    ctx.check(st)
+    return out
+
+
+def _marshal(cands, refs, groups, is_host):
+    n = len(cands)
+    if isinstance(refs, torch.Tensor):
+        refs = [refs] * n
+    if len(refs) != n:
+        raise ValueError("need one reference per candidate tensor, or a single shared one")
+    ptrs = np.empty(n, dtype=np.uint64)
+    descs = np.zeros(n, dtype=_DESC_DTYPE)
+    for i, (c, r) in enumerate(zip(cands, refs)):
+        if c.is_cuda == is_host or r.is_cuda == is_host:
+            raise ValueError("tensor %d lives on the wrong side for this call" % i)
+        if c.dtype != r.dtype or c.numel() != r.numel():
+            raise ValueError("tensor %d: candidate and reference differ in dtype or size" % i)
+        if not (c.is_contiguous() and r.is_contiguous()):
+            raise ValueError("tensor %d must be contiguous" % i)
+        ptrs[i] = c.data_ptr()
+        descs[i] = (c.numel(), r.data_ptr(), dtype_code(c.dtype), 0 if groups is None else int(groups[i]))
+    return ptrs, descs
+
+
+def evo_validate(cands, refs, atol, rtol, groups=None, n_group=0, results=None, group_pass=None, stream=None, ctx=None):
+    """Check CUDA tensors `cands[i]` against `refs[i]` (or one shared tensor).  Returns
+    (results, group_pass): a uint8 CUDA tensor of len(cands) x 40 bytes (evo_result records,
+    see results_to_numpy) and, if `groups` is given, an int32 tensor of n_group verdicts."""
+    n = len(cands)
+    device = cands[0].device if n else torch.device("cuda", torch.cuda.current_device())
+    ctx = ctx or default_context(device.index)
+    ptrs, descs = _marshal(cands, refs, groups, is_host=False)
+    if results is None:
+        results = torch.empty((n, RESULT_DTYPE.itemsize), dtype=torch.uint8, device=device)
+    if groups is not None and group_pass is None:
+        group_pass = torch.empty(int(n_group), dtype=torch.int32, device=device)
+    st = load_library().evo_validate(
+        ctx._h, C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(descs.ctypes.data), n, EVO_F32,
+        float(atol), float(rtol), _dev_ptr(results), _dev_ptr(group_pass) if groups is not None else None,
+        int(n_group) if groups is not None else 0, _stream_ptr(stream, device))
+    ctx.check(st)
+    return results, group_pass
+
+
+def evo_validate_host(cands, refs, atol, rtol, groups=None, n_group=0, device=None, stream=None, ctx=None):
+    """The same check for host tensors (pinned or not): copies, checks and copies the results
+    back inside the library; returns numpy arrays (RESULT_DTYPE records, uint32 verdicts)."""
+    n = len(cands)
+    device = torch.device("cuda", torch.cuda.current_device() if device is None else int(device))
+    ctx = ctx or default_context(device.index)
+    ptrs, descs = _marshal(cands, refs, groups, is_host=True)
+    results = np.zeros(n, dtype=RESULT_DTYPE)
+    gp = np.zeros(int(n_group), dtype=np.uint32) if groups is not None else None
+    st = load_library().evo_validate_host(
+        ctx._h, C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(descs.ctypes.data), n, EVO_F32,
+        float(atol), float(rtol), C.c_void_p(results.ctypes.data),
+        C.c_void_p(gp.ctypes.data) if gp is not None else None, int(n_group) if gp is not None else 0,
+        _stream_ptr(stream, device))
+    ctx.check(st)
+    return results, gp
+
+
+def evo_fitness(times, base_times, passed=None, out=None, stream=None, ctx=None):
+    """times [n_cand, trials] float32 CUDA, base_times [base_trials] float32 CUDA, passed
+    optional int32/uint32 [n_cand].  Returns a uint8 CUDA tensor of n_cand x 16 bytes (evo_fit)."""
+    if times.dtype != torch.float32 or base_times.dtype != torch.float32 or times.dim() != 2:
+        raise ValueError("times must be a 2-D float32 tensor and base_times float32")
+    if not (times.is_contiguous() and base_times.is_contiguous()):
+        raise ValueError("times and base_times must be contiguous")
+    n_cand, trials = times.shape
+    ctx = ctx or default_context(times.device.index)
+    if out is None:
+        out = torch.empty((n_cand, FIT_DTYPE.itemsize), dtype=torch.uint8, device=times.device)
+    st = load_library().evo_fitness(ctx._h, _dev_ptr(times), n_cand, trials, _dev_ptr(base_times), base_times.numel(),
+                                    _dev_ptr(passed), _dev_ptr(out), _stream_ptr(stream, times.device))
+    ctx.check(st)
+    return out
+
+
+def evo_fitness_host(times, base_times, passed=None, device=None, stream=None, ctx=None):
+    """evo_fitness for host arrays (numpy float32); returns a numpy array of FIT_DTYPE records."""
+    times = np.ascontiguousarray(times, dtype=np.float32)
+    base = np.ascontiguousarray(base_times, dtype=np.float32)
+    n_cand, trials = times.shape
+    device = torch.device("cuda", torch.cuda.current_device() if device is None else int(device))
+    ctx = ctx or default_context(device.index)
+    p = np.ascontiguousarray(passed, dtype=np.uint32) if passed is not None else None
+    out = np.zeros(n_cand, dtype=FIT_DTYPE)
+    st = load_library().evo_fitness_host(
+        ctx._h, C.c_void_p(times.ctypes.data), n_cand, trials, C.c_void_p(base.ctypes.data), base.size,
+        C.c_void_p(p.ctypes.data) if p is not None else None, C.c_void_p(out.ctypes.data), _stream_ptr(stream, device))
+    ctx.check(st)
+    return out
+
+
+def results_to_numpy(results):
+    """Device evo_result records -> numpy structured array (synchronises)."""
+    return results.cpu().numpy().view(RESULT_DTYPE).reshape(-1)
+
+
+def fits_to_numpy(fits):
+    return fits.cpu().numpy().view(FIT_DTYPE).reshape(-1)

@@ -1,0 +1,154 @@
+// Context life cycle, error reporting and workspace management of libevo.
+#include <cstdarg>
+#include <cstdio>
+#include <new>
+
+#include "evo_internal.h"
+
+namespace evo {
+
+int fail(evo_ctx* ctx, int status, const char* fmt, ...) {
+    if (ctx) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof buf, fmt, ap);
+        va_end(ap);
+        ctx->last_error = buf;
+    }
+    return status;
+}
+
+int fail_cuda(evo_ctx* ctx, cudaError_t e, const char* what) {
+    return fail(ctx, EVO_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+int reserve_device(evo_ctx* ctx, void** ptr, size_t* have, size_t bytes) {
+    if (*have >= bytes) return EVO_OK;
+    if (*ptr) {
+        // Earlier launches on any stream may still read the old block.
+        EVO_CUDA_TRY(ctx, cudaDeviceSynchronize());
+        EVO_CUDA_TRY(ctx, cudaFree(*ptr));
+        *ptr = nullptr;
+        *have = 0;
+    }
+    size_t want = bytes + bytes / 4;
+    cudaError_t e = cudaMalloc(ptr, want);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        want = bytes;
+        e = cudaMalloc(ptr, want);
+    }
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        *ptr = nullptr;
+        return fail(ctx, EVO_ERR_WORKSPACE, "workspace of %zu bytes: %s", bytes, cudaGetErrorString(e));
+    }
+    *have = want;
+    return EVO_OK;
+}
+
+int reserve_pinned(evo_ctx* ctx, void** ptr, size_t* have, size_t bytes) {
+    if (*have >= bytes) return EVO_OK;
+    if (*ptr) {
+        EVO_CUDA_TRY(ctx, cudaDeviceSynchronize());
+        EVO_CUDA_TRY(ctx, cudaFreeHost(*ptr));
+        *ptr = nullptr;
+        *have = 0;
+    }
+    const size_t want = bytes + bytes / 4;
+    cudaError_t e = cudaMallocHost(ptr, want);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        *ptr = nullptr;
+        return fail(ctx, EVO_ERR_WORKSPACE, "pinned staging of %zu bytes: %s", bytes, cudaGetErrorString(e));
+    }
+    *have = want;
+    return EVO_OK;
+}
+
+DeviceGuard::DeviceGuard(int device) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != device) {
+        err = cudaSetDevice(device);
+        switched = (err == cudaSuccess);
+    }
+}
+
+DeviceGuard::~DeviceGuard() {
+    if (switched) (void)cudaSetDevice(prev);
+}
+
+}  // namespace evo
+
+extern "C" {
+
+int evo_create(evo_ctx** out, int device) {
+    if (!out) return EVO_ERR_ARG;
+    *out = nullptr;
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess || device < 0 || device >= count) {
+        (void)cudaGetLastError();
+        return e != cudaSuccess ? EVO_ERR_CUDA : EVO_ERR_ARG;
+    }
+    evo_ctx* ctx = new (std::nothrow) evo_ctx();
+    if (!ctx) return EVO_ERR_WORKSPACE;
+    ctx->device = device;
+    evo::DeviceGuard guard(device);
+    int status = EVO_OK;
+    if (guard.err != cudaSuccess) status = EVO_ERR_CUDA;
+    if (status == EVO_OK && cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+        status = EVO_ERR_CUDA;
+    if (status == EVO_OK && cudaMalloc(&ctx->d_small, 256) != cudaSuccess) status = EVO_ERR_CUDA;
+    if (status == EVO_OK && cudaEventCreateWithFlags(&ctx->plan_consumed, cudaEventDisableTiming) != cudaSuccess)
+        status = EVO_ERR_CUDA;
+    if (status != EVO_OK) {
+        (void)cudaGetLastError();
+        if (ctx->d_small) (void)cudaFree(ctx->d_small);
+        delete ctx;
+        return status;
+    }
+    *out = ctx;
+    return EVO_OK;
+}
+
+int evo_destroy(evo_ctx* ctx) {
+    if (!ctx) return EVO_OK;
+    evo::DeviceGuard guard(ctx->device);
+    (void)cudaDeviceSynchronize();
+    if (ctx->d_plan) (void)cudaFree(ctx->d_plan);
+    if (ctx->h_plan) (void)cudaFreeHost(ctx->h_plan);
+    if (ctx->d_partials) (void)cudaFree(ctx->d_partials);
+    if (ctx->d_stage) (void)cudaFree(ctx->d_stage);
+    if (ctx->d_small) (void)cudaFree(ctx->d_small);
+    if (ctx->plan_consumed) (void)cudaEventDestroy(ctx->plan_consumed);
+    delete ctx;
+    return EVO_OK;
+}
+
+const char* evo_strerror(int status) {
+    switch (status) {
+        case EVO_OK: return "ok";
+        case EVO_ERR_ARG: return "invalid argument";
+        case EVO_ERR_ALIGN: return "pointer not aligned to its element size";
+        case EVO_ERR_DTYPE: return "unsupported element type";
+        case EVO_ERR_CUDA: return "CUDA runtime error";
+        case EVO_ERR_WORKSPACE: return "workspace unavailable or limit exceeded";
+        case EVO_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+const char* evo_last_error(const evo_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+int evo_set_timing_events(evo_ctx* ctx, void* start, void* stop) {
+    if (!ctx || ((start == nullptr) != (stop == nullptr))) return EVO_ERR_ARG;
+    ctx->time_start = static_cast<cudaEvent_t>(start);
+    ctx->time_stop = static_cast<cudaEvent_t>(stop);
+    return EVO_OK;
+}
+
+uint64_t evo_launch_count(const evo_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

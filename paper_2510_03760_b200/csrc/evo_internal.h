@@ -1,0 +1,54 @@
+// Internal declarations shared by the translation units of libevo (host side).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+
+#include "evo.h"
+
+struct evo_ctx {
+    int device = 0;
+    int sm_count = 0;
+    std::string last_error;
+    uint64_t launches = 0;
+
+    // Scratch owned by the context (see evo.h: grows on demand, freed by evo_destroy).
+    void* d_plan = nullptr;      size_t d_plan_bytes = 0;       // validation plan (device copy)
+    void* h_plan = nullptr;      size_t h_plan_bytes = 0;       // pinned staging of the plan
+    void* d_partials = nullptr;  size_t d_partials_bytes = 0;   // per-(CTA, tensor) partial results
+    void* d_stage = nullptr;     size_t d_stage_bytes = 0;      // tensors of the *_host calls
+    void* d_small = nullptr;                                   // base median, status word
+    cudaEvent_t plan_consumed = nullptr;                       // the last plan upload has been read
+    bool plan_in_flight = false;
+    cudaEvent_t time_start = nullptr, time_stop = nullptr;     // one-shot request of evo_set_timing_events
+};
+
+namespace evo {
+
+int fail(evo_ctx* ctx, int status, const char* fmt, ...);
+int fail_cuda(evo_ctx* ctx, cudaError_t e, const char* what);
+
+// Grows *ptr to at least `bytes` (device memory, contents not preserved).
+int reserve_device(evo_ctx* ctx, void** ptr, size_t* have, size_t bytes);
+int reserve_pinned(evo_ctx* ctx, void** ptr, size_t* have, size_t bytes);
+
+// Sets the context's device for the scope and restores the previous one.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int device);
+    ~DeviceGuard();
+};
+
+inline size_t elem_bytes(int dtype) { return dtype == EVO_F16 || dtype == EVO_BF16 ? 2 : 4; }
+
+}  // namespace evo
+
+#define EVO_CUDA_TRY(ctx, expr)                                            \
+    do {                                                                   \
+        cudaError_t evo_e_ = (expr);                                       \
+        if (evo_e_ != cudaSuccess) return evo::fail_cuda((ctx), evo_e_, #expr); \
+    } while (0)

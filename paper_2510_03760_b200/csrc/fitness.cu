@@ -1,0 +1,146 @@
+// evo_fitness: the performance objective f(p) of the paper's formulation (Section 3.1 Eq. 1):
+// the speedup of a candidate over the baseline kernel (Section 5.1 "Evaluation Metric") from
+// the medians of their run times (Section 4.3: times over repeated runs; Appendix A.7.1: the
+// median of the runs is taken).
+//
+// A few hundred floats per candidate: this is latency, not bandwidth.  One warp owns one row
+// of times in shared memory and selects the middle order statistic(s) by rank counting
+// (rank of x_i = number of j with x_j < x_i, or x_j == x_i and j < i), which needs no sort and
+// is independent of the order in which the trials arrive.
+#include <algorithm>
+
+#include "evo_internal.h"
+
+namespace {
+
+constexpr int kWarpsPerCta = 4;
+constexpr uint32_t kMaxTrials = 4096;
+
+struct RowMedian { float median; uint32_t ok; };
+
+// Median of row[0..trials) held in shared memory, computed by one warp.  ok = 0 when a
+// time is NaN, Inf or not positive.  All lanes return the same value.
+__device__ RowMedian warp_median(const float* row, uint32_t trials, int lane, float* slot /* 2 floats, warp-private */) {
+    const unsigned full = 0xffffffffu;
+    bool bad = false;
+    for (uint32_t i = lane; i < trials; i += 32) {
+        const float x = row[i];
+        bad |= !(x > 0.f && x < __int_as_float(0x7f800000));
+    }
+    if (__any_sync(full, bad)) return RowMedian{0.f, 0u};
+    const uint32_t lo = (trials - 1) / 2, hi = trials / 2;     // equal when trials is odd
+    for (uint32_t i = lane; i < trials; i += 32) {
+        const float x = row[i];
+        uint32_t rank = 0;
+        for (uint32_t j = 0; j < trials; ++j) {
+            const float y = row[j];
+            rank += (y < x || (y == x && j < i)) ? 1u : 0u;
+        }
+        if (rank == lo) slot[0] = x;
+        if (rank == hi) slot[1] = x;
+    }
+    __syncwarp();
+    const float a = slot[0], b = slot[1];
+    __syncwarp();
+    const float med = (lo == hi) ? a : __fmul_rn(0.5f, __fadd_rn(a, b));
+    return RowMedian{med, 1u};
+}
+
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+fitness_kernel(const float* __restrict__ times, uint64_t n_rows, uint32_t trials,
+               const RowMedian* __restrict__ base /* nullptr: write the row's median to base_out */,
+               RowMedian* __restrict__ base_out, const uint32_t* __restrict__ pass, evo_fit* __restrict__ out) {
+    extern __shared__ float smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* row = smem + static_cast<size_t>(warp) * (trials + 2);
+    float* slot = row + trials;
+    const uint64_t r = static_cast<uint64_t>(blockIdx.x) * kWarpsPerCta + warp;
+    if (r >= n_rows) return;
+    const float* src = times + r * trials;
+    for (uint32_t i = lane; i < trials; i += 32) row[i] = src[i];
+    __syncwarp();
+    const RowMedian med = warp_median(row, trials, lane, slot);
+    if (lane != 0) return;
+    if (!base) { *base_out = med; return; }
+    const RowMedian b = *base;
+    evo_fit f;
+    f.median_ms = med.ok ? med.median : 0.f;
+    f.speedup = 0.f;
+    f.valid = 0u;
+    f.status = !med.ok ? 1u : (!b.ok ? 2u : 0u);
+    if (f.status == 0u && (!pass || pass[r] != 0u)) {
+        f.valid = 1u;
+        f.speedup = __fdiv_rn(b.median, med.median);
+    }
+    out[r] = f;
+}
+
+int fitness_device(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
+                   uint32_t base_trials, const uint32_t* pass, evo_fit* out, cudaStream_t stream) {
+    RowMedian* d_base = static_cast<RowMedian*>(ctx->d_small);
+    const size_t smem_base = (static_cast<size_t>(base_trials) + 2) * sizeof(float) * kWarpsPerCta;
+    const size_t smem_rows = (static_cast<size_t>(trials) + 2) * sizeof(float) * kWarpsPerCta;
+    if (std::max(smem_base, smem_rows) > 48 * 1024)
+        EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(fitness_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>((kMaxTrials + 2) * sizeof(float) * kWarpsPerCta)));
+    fitness_kernel<<<1, kWarpsPerCta * 32, smem_base, stream>>>(base_times, 1, base_trials, nullptr, d_base, nullptr, nullptr);
+    ctx->launches += 1;
+    EVO_CUDA_TRY(ctx, cudaGetLastError());
+    if (n_cand == 0) return EVO_OK;
+    const unsigned grid = static_cast<unsigned>((n_cand + kWarpsPerCta - 1) / kWarpsPerCta);
+    fitness_kernel<<<grid, kWarpsPerCta * 32, smem_rows, stream>>>(times, n_cand, trials, d_base, nullptr, pass, out);
+    ctx->launches += 1;
+    EVO_CUDA_TRY(ctx, cudaGetLastError());
+    return EVO_OK;
+}
+
+int check_args(evo_ctx* ctx, const char* who, const float* times, uint64_t n_cand, uint32_t trials,
+               const float* base_times, uint32_t base_trials, evo_fit* out) {
+    if (trials == 0 || base_trials == 0 || trials > kMaxTrials || base_trials > kMaxTrials)
+        return evo::fail(ctx, EVO_ERR_ARG, "%s: trials and base_trials must be in [1, %u]", who, kMaxTrials);
+    if (!base_times || (n_cand > 0 && (!times || !out)))
+        return evo::fail(ctx, EVO_ERR_ARG, "%s: times, base_times and out must not be NULL", who);
+    if (n_cand > (1ull << 31) * kWarpsPerCta) return evo::fail(ctx, EVO_ERR_ARG, "%s: too many candidates", who);
+    if (reinterpret_cast<uintptr_t>(times) % 4 || reinterpret_cast<uintptr_t>(base_times) % 4 || reinterpret_cast<uintptr_t>(out) % 4)
+        return evo::fail(ctx, EVO_ERR_ALIGN, "%s: arrays must be 4-byte aligned", who);
+    return EVO_OK;
+}
+
+}  // namespace
+
+extern "C" int evo_fitness(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
+                           uint32_t base_trials, const uint32_t* pass, evo_fit* out, void* stream) {
+    if (!ctx) return EVO_ERR_ARG;
+    int st = check_args(ctx, "evo_fitness", times, n_cand, trials, base_times, base_trials, out);
+    if (st != EVO_OK) return st;
+    evo::DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
+    return fitness_device(ctx, times, n_cand, trials, base_times, base_trials, pass, out, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int evo_fitness_host(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
+                                uint32_t base_trials, const uint32_t* pass, evo_fit* out, void* stream_) {
+    if (!ctx) return EVO_ERR_ARG;
+    int st = check_args(ctx, "evo_fitness_host", times, n_cand, trials, base_times, base_trials, out);
+    if (st != EVO_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    evo::DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    const size_t b_times = n_cand * trials * sizeof(float), b_base = base_trials * sizeof(float);
+    const size_t o_base = up(b_times), o_pass = o_base + up(b_base), o_out = o_pass + up(n_cand * 4);
+    const size_t total = o_out + up(n_cand * sizeof(evo_fit));
+    st = evo::reserve_device(ctx, &ctx->d_stage, &ctx->d_stage_bytes, std::max<size_t>(total, 256));
+    if (st != EVO_OK) return st;
+    char* base = static_cast<char*>(ctx->d_stage);
+    if (b_times) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(base, times, b_times, cudaMemcpyHostToDevice, stream));
+    EVO_CUDA_TRY(ctx, cudaMemcpyAsync(base + o_base, base_times, b_base, cudaMemcpyHostToDevice, stream));
+    if (pass && n_cand) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(base + o_pass, pass, n_cand * 4, cudaMemcpyHostToDevice, stream));
+    st = fitness_device(ctx, reinterpret_cast<const float*>(base), n_cand, trials, reinterpret_cast<const float*>(base + o_base),
+                        base_trials, pass ? reinterpret_cast<const uint32_t*>(base + o_pass) : nullptr,
+                        reinterpret_cast<evo_fit*>(base + o_out), stream);
+    if (st != EVO_OK) return st;
+    if (n_cand) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(out, base + o_out, n_cand * sizeof(evo_fit), cudaMemcpyDeviceToHost, stream));
+    EVO_CUDA_TRY(ctx, cudaStreamSynchronize(stream));
+    return EVO_OK;
+}

@@ -206,6 +206,12 @@ def special_values(dtype=F32, device="cpu") -> Population:
                       _times(1, 5, 1, device), _times(1, 5, 2, device)[0])
 
 
+def shard_by_candidate(pop: Population, rank: int, world: int) -> List[int]:
+    """Indices of the tensors a replica `rank` of `world` takes when a population is split by
+    candidate id (candidates are independent: no exchange is needed, results concatenate)."""
+    return [i for i, t in enumerate(pop.tensors) if t.group % world == rank]
+
+
 def to_host_bits(t: torch.Tensor):
     """Host numpy view the oracle reads: float32 as is, fp16/bf16 as uint16 bit patterns."""
     t = t.detach().cpu().contiguous()
