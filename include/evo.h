@@ -208,7 +208,7 @@ EVO_API int evo_fitness_host(evo_ctx* ctx, const float* times, uint64_t n_cand, 
  * summary    : host, written.
  * ranges     : host, optional, max_ctas entries; entry b is CTA b's run
  *              [(set_begin, tile_begin), (set_end, tile_end)), tile_end exclusive inside
- *              set_end; set_begin > set_end marks an idle CTA.
+ *              set_end.  Only summary->n_ctas entries are written (runs are never empty).
  * set_of_desc: host, optional, n_desc entries: the set each descriptor joined.
  * set_k      : host, optional, n_desc entries (only the first n_sets are written): members per set.
  * Errors: as evo_validate's argument checks.

@@ -110,7 +110,7 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
     }
     const unsigned __int128 total_cost = prefix[n_sets];
     const uint32_t n_ctas = static_cast<uint32_t>(std::min<uint64_t>(max_ctas, plan->total_tiles));
-    plan->ranges.assign(n_ctas, CtaRange{});
+    plan->ranges.clear();
     plan->n_parts = 0;
     if (n_ctas > 0) {
         // boundary b: the item containing cumulative weight b * total / n_ctas
@@ -134,22 +134,22 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
                 while (p > 0 && tiles[p - 1] == 0) --p;
                 if (p == 0) { se = 0; te = 0; } else { se = p - 1; te = tiles[se]; }
             }
-            const bool empty = sb == n_sets || sb > se || (sb == se && tb >= te);
-            if (empty) {
-                R.s_begin = 1; R.s_end = 0;
-            } else {
-                R.s_begin = sb; R.s_end = se; R.t_begin = tb; R.t_end = te;
-                R.first_member = sets[sb].member_off;
-                R.part_base = plan->n_parts;
-                plan->n_parts += sets[se].member_off + sets[se].k - sets[sb].member_off;
-                for (uint32_t q = sb; q <= se; ++q) {
-                    const uint64_t q0 = q == sb ? tb : 0, q1 = q == se ? te : tiles[q];
-                    if (q0 >= q1) continue;
-                    if (sets[q].cta_first > sets[q].cta_last) sets[q].cta_first = b;
-                    sets[q].cta_last = b;
-                }
+            // Two boundaries can fall into the same item (heavy items, few tiles): such a run
+            // is empty and gets no CTA, so that every CTA in [cta_first, cta_last] of a set
+            // really holds a partial record for it.
+            if (sb == n_sets || sb > se || (sb == se && tb >= te)) continue;
+            const uint32_t cta = static_cast<uint32_t>(plan->ranges.size());
+            R.s_begin = sb; R.s_end = se; R.t_begin = tb; R.t_end = te;
+            R.first_member = sets[sb].member_off;
+            R.part_base = plan->n_parts;
+            plan->n_parts += sets[se].member_off + sets[se].k - sets[sb].member_off;
+            for (uint32_t q = sb; q <= se; ++q) {
+                const uint64_t q0 = q == sb ? tb : 0, q1 = q == se ? te : tiles[q];
+                if (q0 >= q1) continue;
+                if (sets[q].cta_first > sets[q].cta_last) sets[q].cta_first = cta;
+                sets[q].cta_last = cta;
             }
-            plan->ranges[b] = R;
+            plan->ranges.push_back(R);
         }
     }
 

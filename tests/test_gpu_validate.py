@@ -183,9 +183,20 @@ def test_argument_errors(evo):
     with pytest.raises(evo.EvoError) as e:
         evo.evo_validate([c], [r], 0.1, 0.1, groups=[5], n_group=2)
     assert e.value.status == -1
-    with pytest.raises(evo.EvoError) as e:
-        evo.evo_validate([c.view(torch.uint8)[2:6].view(torch.bfloat16)], [r.view(torch.uint8)[1:5].view(torch.bfloat16)], 0.1, 0.1)
-    assert e.value.status == -2
+    # a tensor that is not aligned to its element size (torch cannot build such a view: raw call)
+    import ctypes as C
+    ptrs = np.array([c.data_ptr() + 2], dtype=np.uint64)
+    desc = np.zeros(1, dtype=evo.binding._DESC_DTYPE)
+    desc[0] = (8, r.data_ptr(), evo.EVO_F32, 0)
+    st = L.evo_validate(ctx._h, C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(desc.ctypes.data), 1, evo.EVO_F32,
+                        0.1, 0.1, C.c_void_p(out.data_ptr()), None, 0, None)
+    assert st == -2 and b"aligned" in L.evo_last_error(ctx._h)
+    desc[0] = (8, r.data_ptr(), 9, 0)
+    ptrs[0] = c.data_ptr()
+    assert L.evo_validate(ctx._h, C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(desc.ctypes.data), 1, evo.EVO_F32,
+                          0.1, 0.1, C.c_void_p(out.data_ptr()), None, 0, None) == -3
+    assert L.evo_validate(ctx._h, C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(desc.ctypes.data), 1, evo.EVO_F32,
+                          0.1, 0.1, None, None, 0, None) == -1
     # the context stays usable after errors
     res, _ = evo.evo_validate([c], [r], 0.1, 0.1)
     assert evo.results_to_numpy(res)["pass"][0] == 1

@@ -76,7 +76,7 @@ def test_shared_reference_becomes_one_set_and_cut_is_balanced(lib):
     st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
     assert st == 0 and summ["n_sets"] == 1 and set_k.tolist() == [16] and set(set_of.tolist()) == {0}
     tiles = tiles_of(n, F32, int(summ["tile_bytes"]))
-    assert summ["total_tiles"] == tiles and summ["n_ctas"] == 444
+    assert summ["total_tiles"] == tiles and summ["n_ctas"] == 444 and tiles > 444
     w = coverage(summ, ranges, [tiles])
     assert max(w) - min(w) <= 1
     assert summ["n_parts"] == 444 * 16
@@ -118,7 +118,9 @@ def test_ragged_mixed_population(lib):
             set_tiles[s] = t
             weight_per_tile[s] = int(set_k[s]) + 1
         assert sum(set_k.tolist()) == n_desc
-        assert summ["n_ctas"] == min(max_ctas, sum(set_tiles))
+        assert 0 < summ["n_ctas"] <= min(max_ctas, sum(set_tiles))
+        assert summ["n_ctas"] >= min(max_ctas, sum(set_tiles)) // 2         # few runs are lost to heavy items
+        assert all(r["set_begin"] <= r["set_end"] for r in ranges)          # no idle CTA is launched
         coverage(summ, ranges, set_tiles)
         # weighted balance: no CTA carries more than its share plus one heaviest item
         total = sum(t * w for t, w in zip(set_tiles, weight_per_tile))
@@ -132,6 +134,18 @@ def test_ragged_mixed_population(lib):
                 t1 = int(r["tile_end"]) if s == r["set_end"] else set_tiles[s]
                 wsum += (t1 - t0) * weight_per_tile[s]
             assert wsum <= total / len(ranges) + 2 * heaviest
+
+
+def test_heavy_items_with_few_tiles_leave_no_idle_cta(lib):
+    # 40 members of 3 tiles each: 12 items of very different weight, fewer runs than items
+    descs = np.zeros(80, DESC)
+    descs["n"], descs["dtype"] = 20000, F16
+    descs["ref"][:40], descs["ref"][40:] = 0x7000_0000_0000, 0x7100_0000_0000
+    cands = 0x1000_0000_0000 + np.arange(80, dtype=np.uint64) * 65536
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
+    assert st == 0 and set_k.tolist() == [32, 8, 32, 8] and summ["total_tiles"] == 12
+    assert all(r["set_begin"] <= r["set_end"] for r in ranges) and 0 < summ["n_ctas"] <= 12
+    coverage(summ, ranges, [3, 3, 3, 3])
 
 
 def test_empty_and_zero_length(lib):
