@@ -199,6 +199,43 @@ EVO_API int evo_fitness_host(evo_ctx* ctx, const float* times, uint64_t n_cand, 
                      const uint32_t* pass, evo_fit* out, void* stream);
 
 /*
+ * evo_validate_static - evo_validate for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this entry point exists for the sake of such callers.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a memory pool or a
+ * framework allocator that owns the whole device, under a "no allocation after start-up"
+ * rule of a serving process, or while another part of the program has a CUDA graph capture
+ * open on the thread (an allocation would break the capture).  evo_validate grows its
+ * context's workspace with cudaMalloc when a population needs more room, and creating a
+ * context allocates too; this variant needs no context and never allocates: its scratch
+ * (the schedule and the per-CTA partial results) is a fixed array of 1 MiB that is part of the
+ * library image, so every GPU that loads the library carries that 1 MiB until the process ends.
+ *
+ * Arguments, results, rule and errors are those of evo_validate (all tensor, result and verdict
+ * pointers are device addresses; the caller still provides inputs and outputs), on the CURRENT
+ * device.  Differences:
+ *   - Limit: schedule plus partial results must fit the 1 MiB.  That is roughly 4000 tensors in
+ *     one call (fewer when very many share a reference); the exact need depends on the
+ *     population and is checked per call.  Beyond it the call does nothing and returns
+ *     EVO_ERR_WORKSPACE; evo_validate_static_error() then says how many bytes were needed.
+ *     Split the population over several calls, or use evo_validate.
+ *   - The first call on each device looks up the scratch's device address (no allocation, but a
+ *     runtime query): make that first call before starting any stream capture.
+ *   - All calls on one device share the one scratch array.  It keeps whatever the previous call
+ *     left; nothing in it needs clearing, since each call overwrites every word it later reads.
+ *     But two calls whose kernels overlap on the GPU (different streams, or different threads)
+ *     would overwrite each other's schedule: keep calls on one device ordered, e.g. on one stream.
+ *   - It calls no cudaMalloc, cudaFree, cudaMallocHost nor any other allocating CUDA routine.
+ * evo_validate_static_error: message of the calling thread's last failing evo_validate_static
+ * call ("" if it succeeded); static storage, never NULL.
+ */
+EVO_API int evo_validate_static(const void* const* cand_ptrs /* host array of device ptrs */, const void* ref_ptr /* device */,
+                                const evo_desc* descs /* host */, uint64_t n_desc, int dtype, float atol, float rtol,
+                                evo_result* results /* device */, uint32_t* group_pass /* device, optional */,
+                                uint64_t n_group, void* stream);
+EVO_API const char* evo_validate_static_error(void);
+
+/*
  * evo_plan_inspect - host-only view of the schedule evo_validate would use on a device that
  * runs `max_ctas` persistent CTAs: how descriptors were merged into sets that share one
  * reference read, and which contiguous run of (set, tile) items each CTA walks.  Touches no

@@ -5,6 +5,6 @@ median-of-trials fitness of the EvoEngineer evaluation step, as CUDA kernels beh
 from . import binding  # noqa: F401
 from .binding import (  # noqa: F401
     EVO_U32, EVO_F32, EVO_F16, EVO_BF16, RESULT_DTYPE, FIT_DTYPE, EvoError, Context,
-    evo_gen_inputs, evo_validate, evo_validate_host, evo_fitness, evo_fitness_host,
+    evo_gen_inputs, evo_validate, evo_validate_host, evo_validate_static, evo_fitness, evo_fitness_host,
     default_context, load_library, results_to_numpy, fits_to_numpy, dtype_code,
 )

@@ -54,6 +54,10 @@ def load_library():
         fn = getattr(L, name)
         fn.argtypes = [vp, vp, vp, vp, u64, i32, f32, f32, vp, vp, u64, vp]
         fn.restype = i32
+    L.evo_validate_static.argtypes = [vp, vp, vp, u64, i32, f32, f32, vp, vp, u64, vp]
+    L.evo_validate_static.restype = i32
+    L.evo_validate_static_error.argtypes = []
+    L.evo_validate_static_error.restype = C.c_char_p
     for name in ("evo_fitness", "evo_fitness_host"):
         fn = getattr(L, name)
         fn.argtypes = [vp, vp, u64, u32, vp, u32, vp, vp, vp]
@@ -184,6 +188,25 @@ def evo_validate(cands, refs, atol, rtol, groups=None, n_group=0, results=None, 
         float(atol), float(rtol), _dev_ptr(results), _dev_ptr(group_pass) if groups is not None else None,
         int(n_group) if groups is not None else 0, _stream_ptr(stream, device))
     ctx.check(st)
+    return results, group_pass
+
+
+def evo_validate_static(cands, refs, atol, rtol, results, groups=None, n_group=0, group_pass=None, stream=None):
+    """evo_validate for callers that must not allocate device memory (a process whose allocator
+    owns the device, a no-allocation serving loop): no context, fixed 1 MiB scratch inside the
+    library, current device.  The caller passes the output tensors: `results` (uint8 CUDA,
+    len(cands) x 40 bytes) and, with `groups`, `group_pass` (int32 CUDA, n_group).  Populations
+    that need more scratch than the fixed array raise EvoError (status -5)."""
+    n = len(cands)
+    device = results.device
+    ptrs, descs = _marshal(cands, refs, groups, is_host=False)
+    L = load_library()
+    st = L.evo_validate_static(
+        C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(descs.ctypes.data), n, EVO_F32, float(atol), float(rtol),
+        _dev_ptr(results), _dev_ptr(group_pass) if groups is not None else None,
+        int(n_group) if groups is not None else 0, _stream_ptr(stream, device))
+    if st != 0:
+        raise EvoError(st, "%s (%s)" % (L.evo_strerror(st).decode(), L.evo_validate_static_error().decode()))
     return results, group_pass
 
 

@@ -25,7 +25,10 @@
 
 #include <algorithm>
 #include <cmath>
+#include <cstdarg>
+#include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <unordered_map>
 #include <vector>
@@ -490,5 +493,120 @@ extern "C" int evo_validate_host(evo_ctx* ctx, const void* const* cand_ptrs, con
     if (n_desc) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(results, d_results, n_desc * sizeof(evo_result), cudaMemcpyDeviceToHost, stream));
     if (group_pass) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(group_pass, d_gpass, n_group * sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
     EVO_CUDA_TRY(ctx, cudaStreamSynchronize(stream));
+    return EVO_OK;
+}
+
+// ---- evo_validate_static: the same check without any allocation --------------------------
+//
+// Scratch of the variant below.  It is part of the library image: every GPU that loads the
+// library holds these bytes until the process exits.  In host code `g_static_scratch` is only
+// a stand-in for the symbol; the address a kernel can use comes from cudaGetSymbolAddress.
+constexpr size_t kStaticScratchBytes = 1u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+struct StaticDevice { unsigned char* scratch; int sm_count; bool ready; };
+StaticDevice g_static_dev[kMaxDevices];
+std::mutex g_static_mutex;
+thread_local char g_static_error[256] = "";
+
+int static_fail(int status, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_static_error, sizeof g_static_error, fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+}  // namespace
+
+extern "C" const char* evo_validate_static_error(void) { return g_static_error; }
+
+extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs, uint64_t n_desc,
+                                   int dtype, float atol, float rtol, evo_result* results, uint32_t* group_pass,
+                                   uint64_t n_group, void* stream_) {
+    g_static_error[0] = '\0';
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (n_desc > 0 && !results) return static_fail(EVO_ERR_ARG, "evo_validate_static: results must not be NULL");
+    int device = -1;
+    cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: cudaGetDevice: %s", cudaGetErrorString(e));
+    if (device < 0 || device >= kMaxDevices) return static_fail(EVO_ERR_ARG, "evo_validate_static: device %d out of range", device);
+
+    // Set-up, once per device, with that device current: the device address of the scratch.
+    StaticDevice dev;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_dev[device].ready) {
+            unsigned char* ptr = nullptr;
+            e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_scratch);
+            if (e != cudaSuccess || !ptr)
+                return static_fail(EVO_ERR_CUDA, "evo_validate_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+            int sms = 0;
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+            if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: %s", cudaGetErrorString(e));
+            g_static_dev[device].scratch = ptr;
+            g_static_dev[device].sm_count = sms;
+            g_static_dev[device].ready = true;
+        }
+        dev = g_static_dev[device];
+    }
+
+    Plan plan;
+    std::string err;
+    const uint32_t max_ctas = static_cast<uint32_t>(dev.sm_count) * kCtasPerSm;
+    const int st = build_plan(cand_ptrs, ref_ptr, descs, n_desc, dtype, atol, rtol, group_pass != nullptr, n_group, max_ctas,
+                              &plan, &err);
+    if (st != EVO_OK) return static_fail(st, "evo_validate_static: %s", err.c_str());
+
+    // Layout inside the scratch: the plan, then the partial records.
+    const size_t o_sets = 0;
+    const size_t o_members = align_up(o_sets + plan.sets.size() * sizeof(SetRec), 256);
+    const size_t o_ranges = align_up(o_members + plan.members.size() * sizeof(MemberRec), 256);
+    const size_t o_goff = align_up(o_ranges + plan.ranges.size() * sizeof(CtaRange), 256);
+    const size_t o_gdesc = align_up(o_goff + plan.group_off.size() * 4, 256);
+    const size_t plan_bytes = align_up(o_gdesc + plan.group_desc.size() * 4, 256);
+    const size_t o_parts = plan_bytes;
+    const size_t need = o_parts + static_cast<size_t>(plan.n_parts) * sizeof(Acc);
+    if (need > kStaticScratchBytes)
+        return static_fail(EVO_ERR_WORKSPACE,
+                           "evo_validate_static: this population needs %zu bytes of scratch, the fixed scratch holds %zu "
+                           "(%llu tensors in %zu sets); use evo_validate or split the call",
+                           need, kStaticScratchBytes, (unsigned long long)n_desc, plan.sets.size());
+
+    // The plan goes up from ordinary host memory: the copy call returns once the runtime has
+    // taken the bytes, so the local buffer may go out of scope.
+    std::vector<unsigned char> h(plan_bytes ? plan_bytes : 1);
+    auto put = [&](size_t o, const void* src, size_t bytes) { if (bytes) std::memcpy(h.data() + o, src, bytes); };
+    put(o_sets, plan.sets.data(), plan.sets.size() * sizeof(SetRec));
+    put(o_members, plan.members.data(), plan.members.size() * sizeof(MemberRec));
+    put(o_ranges, plan.ranges.data(), plan.ranges.size() * sizeof(CtaRange));
+    put(o_goff, plan.group_off.data(), plan.group_off.size() * 4);
+    put(o_gdesc, plan.group_desc.data(), plan.group_desc.size() * 4);
+    if (plan_bytes) {
+        e = cudaMemcpyAsync(dev.scratch, h.data(), plan_bytes, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: plan upload: %s", cudaGetErrorString(e));
+    }
+    const unsigned char* d = dev.scratch;
+    const SetRec* d_sets = reinterpret_cast<const SetRec*>(d + o_sets);
+    const MemberRec* d_members = reinterpret_cast<const MemberRec*>(d + o_members);
+    const CtaRange* d_ranges = reinterpret_cast<const CtaRange*>(d + o_ranges);
+    Acc* d_parts = reinterpret_cast<Acc*>(dev.scratch + o_parts);
+    // Nothing in the scratch has to start at zero: pass 1 writes every partial record that
+    // pass 2 reads, so what an earlier call left behind is never looked at.
+    const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
+    if (n_ctas > 0) validate_pass1<<<n_ctas, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol);
+    const uint32_t n_members = static_cast<uint32_t>(n_desc);
+    if (n_members > 0)
+        validate_pass2<<<(n_members + kWarps - 1) / kWarps, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts,
+                                                                                    n_members, results);
+    if (group_pass)
+        group_verdict<<<static_cast<unsigned>((n_group + 255) / 256), 256, 0, stream>>>(
+            reinterpret_cast<const uint32_t*>(d + o_goff), reinterpret_cast<const uint32_t*>(d + o_gdesc), results,
+            static_cast<uint32_t>(n_group), group_pass);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: launch: %s", cudaGetErrorString(e));
     return EVO_OK;
 }
