@@ -40,7 +40,9 @@ WORKLOAD_NOTES = {
 }
 
 
-def build_population(name, device):
+def build_population(name, device, log2_elems=None):
+    if log2_elems is not None:
+        return workloads.config4(device, n=1 << log2_elems)
     return getattr(workloads, name)(device)
 
 
@@ -223,7 +225,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     ctx = evo.Context(local_rank)
-    pop = build_population(args.workload, device)
+    pop = build_population(args.workload, device, args.log2_elems)
     cands = [t.cand for t in pop.tensors]
     refs = [pop.refs[t.ref_index] for t in pop.tensors]
     groups = [t.group for t in pop.tensors]
@@ -381,7 +383,15 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--log2-elems", type=int, default=None,
+                    help="config4 only: shrink every tensor to 2^X elements (a small case for profiler captures; "
+                         "not the benchmark configuration)")
     args = ap.parse_args()
+    if args.log2_elems is not None:
+        if args.workload != "config4" or not 12 <= args.log2_elems <= 28:
+            ap.error("--log2-elems needs --workload config4 and 12 <= X <= 28")
+        args.no_cpu_baseline = True
+        WORKLOAD_NOTES["config4"] = "REDUCED: 16 fp32 candidates x 2^%d elements sharing one reference" % args.log2_elems
     if args.impl == "reference":
         run_reference(args)
     else:
