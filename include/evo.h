@@ -66,7 +66,8 @@ enum { EVO_U32 = 0, EVO_F32 = 1, EVO_F16 = 2, EVO_BF16 = 3 };
 /* Bits of evo_result.flags. */
 enum {
     EVO_FLAG_CAND_NAN = 1, EVO_FLAG_CAND_PINF = 2, EVO_FLAG_CAND_NINF = 4,
-    EVO_FLAG_REF_NAN = 8, EVO_FLAG_REF_INF = 16
+    EVO_FLAG_REF_NAN = 8, EVO_FLAG_REF_INF = 16,
+    EVO_FLAG_INCOMPLETE = 0x40000000   /* the check did not finish (see evo_check); pass is 0, the statistics are 0 */
 };
 
 typedef struct evo_ctx evo_ctx;
@@ -250,7 +251,7 @@ EVO_API const char* evo_validate_static_error(void);
  * set_k      : host, optional, n_desc entries (only the first n_sets are written): members per set.
  * Errors: as evo_validate's argument checks.
  */
-typedef struct { uint32_t n_sets, n_ctas, n_parts, tile_bytes; uint64_t total_tiles; } evo_plan_summary;
+typedef struct { uint32_t n_sets, n_ctas, n_parts, tile_elems; uint64_t total_tiles; } evo_plan_summary;
 typedef struct { uint64_t tile_begin, tile_end; uint32_t set_begin, set_end; } evo_plan_range;
 EVO_API int evo_plan_inspect(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs, uint64_t n_desc,
                              int dtype, uint32_t max_ctas, evo_plan_summary* summary, evo_plan_range* ranges,
@@ -265,6 +266,17 @@ EVO_API int evo_plan_inspect(const void* const* cand_ptrs, const void* ref_ptr, 
  * no counterpart.)
  */
 EVO_API int evo_set_timing_events(evo_ctx* ctx, void* start, void* stop);
+
+/*
+ * evo_check - wait for the work enqueued on `stream` and report whether the device side of
+ * the context's calls ran to completion.  The kernels never wait without a limit (a copy
+ * into shared memory that does not land within 2 s makes the CTA stop, raise a status word
+ * and return); when that happened, evo_validate's results carry EVO_FLAG_INCOMPLETE with
+ * pass = 0, and this call returns EVO_ERR_TIMEOUT once and clears the word.  The *_host
+ * variants do this check themselves.  (The paper has no counterpart.)
+ * Errors: EVO_ERR_ARG, EVO_ERR_CUDA, EVO_ERR_TIMEOUT.
+ */
+EVO_API int evo_check(evo_ctx* ctx, void* stream);
 
 /* Number of kernels this context has launched so far (for accounting in benchmarks). */
 EVO_API uint64_t evo_launch_count(const evo_ctx* ctx);

@@ -48,6 +48,8 @@ def load_library():
     L.evo_launch_count.restype = u64
     L.evo_set_timing_events.argtypes = [vp, vp, vp]
     L.evo_set_timing_events.restype = i32
+    L.evo_check.argtypes = [vp, vp]
+    L.evo_check.restype = i32
     L.evo_gen_inputs.argtypes = [vp, u64, u64, i32, u64, vp, vp]
     L.evo_gen_inputs.restype = i32
     for name in ("evo_validate", "evo_validate_host"):
@@ -95,6 +97,10 @@ class Context:
             self._h, C.c_void_p(start.cuda_event) if start is not None else None,
             C.c_void_p(stop.cuda_event) if stop is not None else None)
         self.check(st)
+
+    def synchronize(self, stream=None):
+        """evo_check: wait for `stream` and raise EvoError(-6) if a device-side wait ran out."""
+        self.check(load_library().evo_check(self._h, _stream_ptr(stream, torch.device("cuda", self.device))))
 
     def close(self):
         if self._h is not None and _lib is not None:

@@ -79,6 +79,15 @@ DeviceGuard::~DeviceGuard() {
     if (switched) (void)cudaSetDevice(prev);
 }
 
+int sync_and_check(evo_ctx* ctx, cudaStream_t stream, const char* who) {
+    EVO_CUDA_TRY(ctx, cudaStreamSynchronize(stream));
+    uint32_t word = 0;
+    EVO_CUDA_TRY(ctx, cudaMemcpy(&word, status_word(ctx), sizeof word, cudaMemcpyDeviceToHost));
+    if (word == 0) return EVO_OK;
+    EVO_CUDA_TRY(ctx, cudaMemset(status_word(ctx), 0, sizeof word));
+    return fail(ctx, EVO_ERR_TIMEOUT, "%s: a device-side wait ran out (status word 0x%x); results are marked incomplete", who, word);
+}
+
 }  // namespace evo
 
 extern "C" {
@@ -101,6 +110,7 @@ int evo_create(evo_ctx** out, int device) {
     if (status == EVO_OK && cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
         status = EVO_ERR_CUDA;
     if (status == EVO_OK && cudaMalloc(&ctx->d_small, 256) != cudaSuccess) status = EVO_ERR_CUDA;
+    if (status == EVO_OK && cudaMemset(ctx->d_small, 0, 256) != cudaSuccess) status = EVO_ERR_CUDA;
     if (status == EVO_OK && cudaEventCreateWithFlags(&ctx->plan_consumed, cudaEventDisableTiming) != cudaSuccess)
         status = EVO_ERR_CUDA;
     if (status != EVO_OK) {
@@ -147,6 +157,13 @@ int evo_set_timing_events(evo_ctx* ctx, void* start, void* stop) {
     ctx->time_start = static_cast<cudaEvent_t>(start);
     ctx->time_stop = static_cast<cudaEvent_t>(stop);
     return EVO_OK;
+}
+
+int evo_check(evo_ctx* ctx, void* stream) {
+    if (!ctx) return EVO_ERR_ARG;
+    evo::DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
+    return evo::sync_and_check(ctx, static_cast<cudaStream_t>(stream), "evo_check");
 }
 
 uint64_t evo_launch_count(const evo_ctx* ctx) { return ctx ? ctx->launches : 0; }

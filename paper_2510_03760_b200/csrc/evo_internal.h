@@ -19,7 +19,8 @@ struct evo_ctx {
     void* h_plan = nullptr;      size_t h_plan_bytes = 0;       // pinned staging of the plan
     void* d_partials = nullptr;  size_t d_partials_bytes = 0;   // per-(CTA, tensor) partial results
     void* d_stage = nullptr;     size_t d_stage_bytes = 0;      // tensors of the *_host calls
-    void* d_small = nullptr;                                   // base median, status word
+    void* d_small = nullptr;                                   // 256 bytes: baseline median (0..127), status word (128)
+    bool pass1_ready = false;                                  // the first pass's shared-memory size has been set
     cudaEvent_t plan_consumed = nullptr;                       // the last plan upload has been read
     bool plan_in_flight = false;
     cudaEvent_t time_start = nullptr, time_stop = nullptr;     // one-shot request of evo_set_timing_events
@@ -42,6 +43,11 @@ struct DeviceGuard {
     explicit DeviceGuard(int device);
     ~DeviceGuard();
 };
+
+// Device word that a kernel raises when one of its bounded waits ran out.
+inline uint32_t* status_word(evo_ctx* ctx) { return reinterpret_cast<uint32_t*>(static_cast<char*>(ctx->d_small) + 128); }
+// Synchronises `stream`, then reads and clears the status word: EVO_OK or EVO_ERR_TIMEOUT.
+int sync_and_check(evo_ctx* ctx, cudaStream_t stream, const char* who);
 
 inline size_t elem_bytes(int dtype) { return dtype == EVO_F16 || dtype == EVO_BF16 ? 2 : 4; }
 

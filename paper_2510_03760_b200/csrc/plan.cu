@@ -104,7 +104,7 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
     prefix[0] = 0;
     plan->total_tiles = 0;
     for (uint32_t s = 0; s < n_sets; ++s) {
-        tiles[s] = (sets[s].n + tile_elems(sets[s].dtype) - 1) / tile_elems(sets[s].dtype);
+        tiles[s] = (sets[s].n + kTileElems - 1) / kTileElems;
         plan->total_tiles += tiles[s];
         prefix[s + 1] = prefix[s] + static_cast<unsigned __int128>(tiles[s]) * (sets[s].k + 1);
     }
@@ -182,7 +182,7 @@ extern "C" EVO_API int evo_plan_inspect(const void* const* cand_ptrs, const void
     summary->n_sets = static_cast<uint32_t>(plan.sets.size());
     summary->n_ctas = static_cast<uint32_t>(plan.ranges.size());
     summary->n_parts = plan.n_parts;
-    summary->tile_bytes = evo::kTileBytes;
+    summary->tile_elems = evo::kTileElems;
     summary->total_tiles = plan.total_tiles;
     if (ranges) {
         for (size_t b = 0; b < plan.ranges.size(); ++b) {

@@ -12,12 +12,12 @@
 
 namespace evo {
 
-constexpr int kThreads = 256;                   // threads per CTA of the validation kernels
+constexpr int kThreads = 256;                   // consumer threads per CTA of the first pass (8 warps)
 constexpr int kWarps = kThreads / 32;
+constexpr int kBlock = kThreads + 32;           // plus one producer warp that issues the bulk copies
 constexpr int kMaxK = 32;                       // members of one set (more are split into several sets)
-constexpr int kVpt = 4;                         // 16-byte vectors per thread per tile
-constexpr int kTileVecs = kVpt * kThreads;      // 16-byte vectors per tile
-constexpr int kTileBytes = kTileVecs * 16;      // 16 KiB of every tensor per tile
+constexpr int kEpt = 16;                        // elements per consumer thread per tile
+constexpr int kTileElems = kEpt * kThreads;     // 4096 elements of every tensor per tile (16 KiB fp32, 8 KiB fp16/bf16)
 
 struct Acc {                 // partial result of one tensor (40 bytes)
     unsigned long long mism;
@@ -54,11 +54,6 @@ struct CtaRange {            // items [(s_begin, t_begin), (s_end, t_end)) with 
     uint32_t part_base;      // first partial record of this CTA
     uint32_t first_member;   // member_off of s_begin
 };
-
-#if defined(__CUDACC__)
-__host__ __device__
-#endif
-inline uint64_t tile_elems(uint32_t dtype) { return dtype == EVO_F32 ? kTileBytes / 4 : kTileBytes / 2; }
 
 struct Plan {
     std::vector<SetRec> sets;

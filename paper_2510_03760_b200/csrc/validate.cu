@@ -3,23 +3,30 @@
 // reference outputs), with the error statistics reported alongside the verdict.
 //
 // Shape of the computation: a pure streaming read.  Every candidate element and every
-// distinct reference element has to come from HBM once; per element there are about ten
-// binary32 operations.  The design therefore spends its effort on (1) never reading a
+// distinct reference element has to come from HBM once; per element there are seven to
+// nine binary32 operations.  The design therefore spends its effort on (1) never reading a
 // reference tile more than once per set of candidates that share it, (2) keeping many
-// 16-byte loads in flight per SM, and (3) keeping reductions off the per-element path.
+// bytes in flight per SM independently of the arithmetic, and (3) keeping reductions and
+// everything that depends on the reference alone off the per-candidate path.
 //
 //   plan (host)   tensors with the same (reference, n, dtype) form a set of up to kMaxK
-//                 members; the flat list of (set, tile) items, weighted by the bytes they
+//                 members; the flat list of (set, tile) items, weighted by the tiles they
 //                 move, is cut into one contiguous range per CTA (a fixed cut: no work
 //                 queue, no atomics, results reproducible run to run).
-//   pass 1        persistent CTAs walk their range.  Per tile the reference is loaded
-//                 once into registers (128-bit loads) and compared against each member's
-//                 tile; per (tile, member) the warp folds its lanes with redux/shuffles
-//                 into a warp-private accumulator in shared memory.  When a CTA leaves a
-//                 set it writes one partial record per member to global memory.
+//   pass 1        persistent CTAs walk their range.  A producer warp streams the tiles
+//                 (reference, then each member) into a ring of shared-memory stages with
+//                 bulk asynchronous copies that complete on mbarriers; eight consumer warps
+//                 take a reference tile into registers once (value, tolerance, |r|), then
+//                 compare each member's tile against it.  Per (tile, member) a warp folds
+//                 its lanes with redux/shuffles into a warp-private accumulator in shared
+//                 memory.  When a CTA leaves a set it writes one partial record per member.
 //   pass 2        one warp per tensor folds the partial records of the CTAs that touched
 //                 it, in a fixed order, and writes the evo_result.
 //   verdict       one thread per candidate id ANDs the verdicts of its tensors.
+//
+// Every wait on an mbarrier is bounded: after kWaitLimitNs the CTA stops working, lets its
+// outstanding copies land, raises the status word and returns; pass 2 then marks every
+// result as incomplete instead of reporting numbers.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -40,15 +47,91 @@ namespace {
 
 using namespace evo;
 
-constexpr int kCtasPerSm = 3;
+constexpr int kCtasPerSm = 2;
+constexpr int kStages = 6;                          // ring depth per CTA
+constexpr int kStageBytes = kTileElems * 4;         // 16 KiB: one fp32 tile (a 16-bit tile uses half)
+constexpr size_t kRingBytes = static_cast<size_t>(kStages) * kStageBytes;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, then give up
 
-// ---- loads ---------------------------------------------------------------------------
-// Streaming 128-bit load: the data is used exactly once by this SM.
-__device__ __forceinline__ uint4 load_stream(const uint4* p) { return __ldcs(p); }
+// ---- shared-memory barriers and bulk copies (PTX) -------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait, cold part: polls until the phase completes, another warp of the CTA has given
+// up, or the limit has passed (then raises the CTA's abort flag itself).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag);
+}
+__device__ __forceinline__ unsigned long long policy_evict_first() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// One contiguous block global -> this CTA's shared memory; completion is counted in bytes on
+// `bar`.  Source, destination and size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, unsigned long long pol) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+
+// Position in the ring: both the producer and the consumers count the same sequence of tiles.
+struct Ring {
+    uint32_t full0, empty0;     // shared-memory addresses of full[0], empty[0]
+    uint32_t data0;             // ... and of stage 0
+    uint32_t stage = 0, phase = 0;
+    bool dead = false;          // this warp has given up (warp-uniform)
+    volatile int* abort_flag;
+    __device__ __forceinline__ uint32_t full() const { return full0 + 8u * stage; }
+    __device__ __forceinline__ uint32_t empty() const { return empty0 + 8u * stage; }
+    __device__ __forceinline__ uint32_t data() const { return data0 + static_cast<uint32_t>(kStageBytes) * stage; }
+    __device__ __forceinline__ void advance() { if (++stage == kStages) { stage = 0; phase ^= 1u; } }
+};
+
+// ---- element types ---------------------------------------------------------------------
 template <int DT> struct Elem;
 template <> struct Elem<EVO_F32> {
     static constexpr int kPerVec = 4;
+    static constexpr int kVecs = kEpt / 4;          // 16-byte vectors per thread per tile
     using T = float;
     static __device__ __forceinline__ float at(const uint4& v, int i) {
         return __uint_as_float(i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w);
@@ -57,6 +140,7 @@ template <> struct Elem<EVO_F32> {
 };
 template <> struct Elem<EVO_F16> {
     static constexpr int kPerVec = 8;
+    static constexpr int kVecs = kEpt / 8;
     using T = __half;
     static __device__ __forceinline__ float at(const uint4& v, int i) {
         const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
@@ -67,6 +151,7 @@ template <> struct Elem<EVO_F16> {
 };
 template <> struct Elem<EVO_BF16> {
     static constexpr int kPerVec = 8;
+    static constexpr int kVecs = kEpt / 8;
     using T = __nv_bfloat16;
     static __device__ __forceinline__ float at(const uint4& v, int i) {
         const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
@@ -75,37 +160,20 @@ template <> struct Elem<EVO_BF16> {
     static __device__ __forceinline__ float widen(T x) { return __bfloat162float(x); }
 };
 
-// ---- per-lane state for one (tile, member) ----------------------------------------------
+// ---- the rule, exact form ----------------------------------------------------------------
+// Per-lane state for one (tile, member) on the exact path.
 struct Lane {
     uint32_t cnt = 0;        // mismatches
     float ma = 0.f;          // max d
-    float mr = 0.f;          // max d/|r| found by this lane (exact path only)
-    float sse = 0.f;         // sum d^2, binary32 (fast path)
-    double dsse = 0.0;       // sum d^2, binary64 (exact path)
+    float mr = 0.f;          // max d/|r|
+    double dsse = 0.0;       // sum d^2, binary64
     uint32_t nf = 0;         // non-finite elements
     uint32_t flags = 0;
-    bool trig = false;       // some quotient may exceed the running maximum
-    bool exact = false;      // values above come from the exact path
 };
 
-// Fast path, valid when c and r are finite and d does not overflow.  Operations and
-// rounding follow the rule literally: d = |c - r|, tol = atol + rtol*|r|, no fused
-// multiply-add on that chain.  With atol, rtol >= 0 and finite data, c == r implies
-// d = 0 <= tol, so the equality clause needs no separate test here.
-// The quotient d/|r| is not formed: `mlo` is a value slightly below the running maximum m
-// of the quotient, and d > RZ(mlo*|r|) holds whenever fl(d/|r|) > m could (rounding the
-// product toward zero keeps the test one-sided), so a miss never loses a maximum.
-__device__ __forceinline__ void fast_elem(float c, float r, float atol, float rtol, float mlo, Lane& s) {
-    const float d = fabsf(__fsub_rn(c, r));
-    const float ar = fabsf(r);
-    const float tol = __fadd_rn(atol, __fmul_rn(rtol, ar));
-    s.cnt += (d > tol) ? 1u : 0u;
-    s.ma = fmaxf(s.ma, d);
-    s.sse = fmaf(d, d, s.sse);
-    s.trig |= (d > __fmul_rz(mlo, ar));
-}
-
-// Exact path: the rule with every special case, and the true quotient.
+// The rule with every special case, and the true quotient: d = |c - r|, tol = atol + rtol*|r|
+// (one rounding per operation, no fused multiply-add), close = (c == r) or (d finite and
+// d <= tol); NaN/Inf elements are counted and flagged and stay out of the statistics.
 __device__ __forceinline__ void exact_elem(float c, float r, float atol, float rtol, Lane& s) {
     const float d = fabsf(__fsub_rn(c, r));
     const float ar = fabsf(r);
@@ -131,170 +199,347 @@ __device__ __forceinline__ void exact_elem(float c, float r, float atol, float r
     }
 }
 
-// Fold the 32 lanes and add the result to the warp's accumulator for this member.
-__device__ __forceinline__ void warp_commit(const Lane& s, Acc* acc, int lane) {
+// Fold the 32 lanes (all fields) and add the result to the warp's accumulator for this member.
+__device__ __forceinline__ void warp_commit_exact(const Lane& s, Acc* acc, int lane) {
     const unsigned full = 0xffffffffu;
     const uint32_t cnt = __reduce_add_sync(full, s.cnt);
     const uint32_t ma = __reduce_max_sync(full, __float_as_uint(s.ma));
-    const bool any_exact = __any_sync(full, s.exact);
-    double sse;
-    uint32_t mr = 0, nf = 0, fl = 0;
-    if (any_exact) {
-        double x = s.exact ? s.dsse : static_cast<double>(s.sse);
+    const uint32_t mr = __reduce_max_sync(full, __float_as_uint(s.mr));
+    const uint32_t nf = __reduce_add_sync(full, s.nf);
+    const uint32_t fl = __reduce_or_sync(full, s.flags);
+    double x = s.dsse;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(full, x, o);
-        sse = x;
-        mr = __reduce_max_sync(full, __float_as_uint(s.mr));
-        nf = __reduce_add_sync(full, s.nf);
-        fl = __reduce_or_sync(full, s.flags);
-    } else {
-        float x = s.sse;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(full, x, o);
-        sse = static_cast<double>(x);
-    }
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(full, x, o);
     if (lane == 0) {
         acc->mism += cnt;
-        acc->sse += sse;
+        acc->nonfin += nf;
+        acc->sse += x;
         acc->max_abs = max(acc->max_abs, ma);
-        if (any_exact) {
-            acc->nonfin += nf;
-            acc->max_rel = max(acc->max_rel, mr);
-            acc->flags |= fl;
-        }
+        acc->max_rel = max(acc->max_rel, mr);
+        acc->flags |= fl;
     }
     __syncwarp();
 }
 
-// The exact path over this thread's share of a full tile.  Reached rarely (first tile of a
-// set, a new maximum of the quotient, NaN/Inf, overflow or all-tiny differences), so it
-// re-reads its 16-byte vectors (they were just loaded: L2 hits) instead of holding the hot
-// loop's registers hostage.
+// The exact rule over this thread's 16 elements of a full tile, read again from global
+// memory (they were just streamed: L2 hits at best).  Reached only when the fast path
+// cannot vouch for its numbers: a NaN/Inf, an overflowing difference, or differences so
+// small that their squares underflow in binary32.
 template <int DT>
 __device__ __noinline__ void exact_redo(const uint4* __restrict__ cp, const uint4* __restrict__ rp,
-                                        float atol, float rtol, Lane& st) {
+                                        float atol, float rtol, Lane* out) {
     using E = Elem<DT>;
-    st = Lane();
-    st.exact = true;
+    Lane st;
 #pragma unroll 1
-    for (int v = 0; v < kVpt; ++v) {
+    for (int v = 0; v < E::kVecs; ++v) {
         const uint4 c = cp[v * kThreads], r = rp[v * kThreads];
 #pragma unroll
         for (int e = 0; e < E::kPerVec; ++e) exact_elem(E::at(c, e), E::at(r, e), atol, rtol, st);
     }
+    *out = st;
 }
 
+// ---- consumers ---------------------------------------------------------------------------
+// Wait until the producer's copy into the current stage has landed.  The answer is the same
+// for all lanes of the warp; after a failed wait the warp does no further work.
+__device__ __forceinline__ bool ring_acquire(Ring& g) {
+    const bool ok = mbar_wait(g.full(), g.phase, g.abort_flag);
+    if (!__all_sync(0xffffffffu, ok)) { g.dead = true; return false; }
+    return true;
+}
+// The warp has copied its share of the stage into registers: hand the stage back.
+__device__ __forceinline__ void ring_release(Ring& g, int lane) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(g.empty());
+    g.advance();
+}
+
+constexpr float kInf = __builtin_huge_valf();
+constexpr float kShrink = 0.99999904632568359375f;      // 1 - 2^-20
+
 // One full, 16-byte aligned tile: reference into registers once, then every member.
+//
+// Fast path per element, valid when c and r are finite and d does not overflow:
+// d = |c - r| against the tolerance computed once per reference element; with atol, rtol >= 0
+// and finite data c == r implies d = 0 <= tol, so the equality clause needs no test here.
+// The quotient d/|r| is not formed: `mlo` is slightly below the running maximum m of the
+// quotient, and d > RZ(mlo*|r|) holds whenever fl(d/|r|) > m could (rounding the product
+// toward zero keeps the test one-sided), so a miss never loses a maximum.  A thread whose
+// filter fired walks its 16 elements again in registers and divides only where r != 0 and
+// the filter still fires against its own, rising maximum.
 template <int DT>
 __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float atol, float rtol,
-                                          Acc (*s_acc)[kWarps], const void* const* s_cand, int warp, int lane) {
+                                          Acc (*s_acc)[kWarps], const void* const* s_cand, Ring& g, int warp, int lane) {
     using E = Elem<DT>;
-    const uint64_t base = t * kTileVecs + threadIdx.x;
-    const uint4* rp = static_cast<const uint4*>(S.ref) + base;
-    uint4 r[kVpt];
+    if (g.dead) return;
+    constexpr uint32_t kVecStride = kThreads * 16;
+    float r[kEpt], tol[kEpt];
+    if (!ring_acquire(g)) return;
+    {
+        const uint32_t a = g.data() + threadIdx.x * 16;
 #pragma unroll
-    for (int v = 0; v < kVpt; ++v) r[v] = load_stream(rp + v * kThreads);
+        for (int v = 0; v < E::kVecs; ++v) {
+            const uint4 x = lds128(a + v * kVecStride);
+#pragma unroll
+            for (int e = 0; e < E::kPerVec; ++e) r[v * E::kPerVec + e] = E::at(x, e);
+        }
+    }
+    ring_release(g, lane);
+#pragma unroll
+    for (int e = 0; e < kEpt; ++e) tol[e] = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r[e])));
+    const uint64_t vec0 = t * (kTileElems / E::kPerVec) + threadIdx.x;   // this thread's first vector of the tile
     const int K = static_cast<int>(S.k);
 #pragma unroll 1
     for (int k = 0; k < K; ++k) {
-        const uint4* cp = static_cast<const uint4*>(s_cand[k]) + base;
-        uint4 c[kVpt];
+        if (!ring_acquire(g)) return;
+        uint4 cv[E::kVecs];
+        {
+            const uint32_t a = g.data() + threadIdx.x * 16;
 #pragma unroll
-        for (int v = 0; v < kVpt; ++v) c[v] = load_stream(cp + v * kThreads);
+            for (int v = 0; v < E::kVecs; ++v) cv[v] = lds128(a + v * kVecStride);
+        }
+        ring_release(g, lane);
         Acc* acc = &s_acc[k][warp];
         const float m = __uint_as_float(acc->max_rel);
-        const float mlo = __fmul_rz(m, 0.99999904632568359375f);      // 1 - 2^-20
-        Lane st;
+        const float mlo = __fmul_rz(m, kShrink);
+        uint32_t cnt = 0;
+        float ma = 0.f, sse = 0.f;
+        bool trig = false;
 #pragma unroll
-        for (int v = 0; v < kVpt; ++v)
+        for (int v = 0; v < E::kVecs; ++v)
 #pragma unroll
-            for (int e = 0; e < E::kPerVec; ++e) fast_elem(E::at(c[v], e), E::at(r[v], e), atol, rtol, mlo, st);
-        // Leave the fast path if (a) something was NaN/Inf or overflowed (the sum of squares
-        // is then NaN/Inf), (b) a quotient may beat the running maximum, or (c) every d is so
-        // small that d^2 underflows in binary32.
-        const bool redo = !(st.sse < __int_as_float(0x7f800000)) || st.trig ||
-                          (st.ma < 9.094947017729282e-13f /* 2^-40 */ && st.ma > 0.f);
-        if (redo) exact_redo<DT>(cp, rp, atol, rtol, st);
-        warp_commit(st, acc, lane);
+            for (int e = 0; e < E::kPerVec; ++e) {
+                const int i = v * E::kPerVec + e;
+                const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
+                cnt += (d > tol[i]) ? 1u : 0u;
+                ma = fmaxf(ma, d);
+                sse = fmaf(d, d, sse);
+                trig |= d > __fmul_rz(mlo, fabsf(r[i]));
+            }
+        // The fast numbers do not stand if something was NaN/Inf or overflowed (the sum of
+        // squares is then NaN/Inf) or if every d is so small that d^2 underflows in binary32.
+        const bool redo = !(sse < kInf) || (ma < 9.094947017729282e-13f /* 2^-40 */ && ma > 0.f);
+        float mt = m;
+        if (trig && !redo) {
+            float lo = mlo;
+#pragma unroll
+            for (int v = 0; v < E::kVecs; ++v)
+#pragma unroll
+                for (int e = 0; e < E::kPerVec; ++e) {
+                    const int i = v * E::kPerVec + e;
+                    const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
+                    const float ar = fabsf(r[i]);
+                    if (ar != 0.f && d > __fmul_rz(lo, ar)) {
+                        const float q = __fdiv_rn(d, ar);
+                        if (q > mt) { mt = q; lo = __fmul_rz(mt, kShrink); }
+                    }
+                }
+        }
+        const unsigned full = 0xffffffffu;
+        if (__any_sync(full, redo)) {
+            Lane st;
+            if (redo) {
+                exact_redo<DT>(static_cast<const uint4*>(s_cand[k]) + vec0, static_cast<const uint4*>(S.ref) + vec0,
+                               atol, rtol, &st);
+            } else {
+                st.cnt = cnt; st.ma = ma; st.mr = mt; st.dsse = static_cast<double>(sse);
+            }
+            warp_commit_exact(st, acc, lane);
+        } else {
+            const uint32_t cnt_w = __reduce_add_sync(full, cnt);
+            const uint32_t ma_w = __reduce_max_sync(full, __float_as_uint(ma));
+            const uint32_t mr_w = __reduce_max_sync(full, __float_as_uint(mt));
+            float x = sse;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(full, x, o);
+            if (lane == 0) {
+                acc->mism += cnt_w;
+                acc->sse += static_cast<double>(x);
+                acc->max_abs = max(acc->max_abs, ma_w);
+                acc->max_rel = max(acc->max_rel, mr_w);
+            }
+            __syncwarp();
+        }
     }
 }
 
-// Ragged last tile, or tensors that are not 16-byte aligned: scalar loads, exact path.
+// Ragged last tile, or tensors that are not 16-byte aligned: scalar loads straight from
+// global memory, exact rule.  These tiles do not pass through the ring.
 template <int DT>
 __device__ __noinline__ void slow_tile(const SetRec& S, uint64_t t, float atol, float rtol,
                                        Acc (*s_acc)[kWarps], const void* const* s_cand, int warp, int lane) {
     using E = Elem<DT>;
     using T = typename E::T;
-    const uint64_t e0 = t * tile_elems(DT);
-    const uint64_t e1 = min(S.n, e0 + tile_elems(DT));
+    const uint64_t e0 = t * kTileElems;
+    const uint64_t e1 = min(S.n, e0 + kTileElems);
     const T* rp = static_cast<const T*>(S.ref);
     for (uint32_t k = 0; k < S.k; ++k) {
         const T* cp = static_cast<const T*>(s_cand[k]);
         Lane st;
-        st.exact = true;
         for (uint64_t e = e0 + threadIdx.x; e < e1; e += kThreads) exact_elem(E::widen(cp[e]), E::widen(rp[e]), atol, rtol, st);
-        warp_commit(st, &s_acc[k][warp], lane);
+        warp_commit_exact(st, &s_acc[k][warp], lane);
     }
+}
+
+// Tiles of set s that belong to this CTA's range, and how many of the set's tiles are full
+// and aligned (those travel through the ring; producer and consumers must agree on this).
+__device__ __forceinline__ void set_span(const CtaRange& rg, uint32_t s, const SetRec& S, uint64_t* t0, uint64_t* t1,
+                                         uint64_t* ring_tiles) {
+    const uint64_t tiles = (S.n + kTileElems - 1) / kTileElems;
+    *t0 = (s == rg.s_begin) ? rg.t_begin : 0;
+    *t1 = (s == rg.s_end) ? rg.t_end : tiles;
+    *ring_tiles = S.vec_ok ? S.n / kTileElems : 0;
 }
 
 template <int DT>
-__device__ __forceinline__ void run_set(const SetRec& S, uint64_t t0, uint64_t t1, float atol, float rtol,
-                                        Acc (*s_acc)[kWarps], const void* const* s_cand, int warp, int lane) {
-    const uint64_t full_tiles = S.vec_ok ? S.n / tile_elems(DT) : 0;
+__device__ __forceinline__ void run_set(const SetRec& S, uint64_t t0, uint64_t t1, uint64_t ring_tiles, float atol, float rtol,
+                                        Acc (*s_acc)[kWarps], const void* const* s_cand, Ring& g, int warp, int lane) {
     for (uint64_t t = t0; t < t1; ++t) {
-        if (t < full_tiles) fast_tile<DT>(S, t, atol, rtol, s_acc, s_cand, warp, lane);
-        else slow_tile<DT>(S, t, atol, rtol, s_acc, s_cand, warp, lane);
+        if (t < ring_tiles) fast_tile<DT>(S, t, atol, rtol, s_acc, s_cand, g, warp, lane);
+        else if (!g.dead) slow_tile<DT>(S, t, atol, rtol, s_acc, s_cand, warp, lane);
     }
 }
 
-__global__ void __launch_bounds__(kThreads, kCtasPerSm)
+// ---- producer ----------------------------------------------------------------------------
+// One warp walks the CTA's range ahead of the consumers and fills the ring: per tile the
+// reference, then each member.  Lane k keeps member k's base address; lane 0 waits for the
+// stage to be free, arms its barrier with the byte count and issues the copy.
+// Returns how many copies were issued.
+__device__ __forceinline__ uint32_t producer_loop(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
+                                                  const CtaRange& rg, Ring& g, int lane) {
+    const unsigned full = 0xffffffffu;
+    const unsigned long long pol = policy_evict_first();
+    uint32_t issued = 0;
+    for (uint32_t s = rg.s_begin; s <= rg.s_end && !g.dead; ++s) {
+        const SetRec S = sets[s];
+        uint64_t t0, t1, ring_tiles;
+        set_span(rg, s, S, &t0, &t1, &ring_tiles);
+        if (t1 > ring_tiles) t1 = ring_tiles;
+        if (t0 >= t1) continue;
+        const uint32_t tile_bytes = kTileElems * (S.dtype == EVO_F32 ? 4u : 2u);
+        const unsigned long long mine = (static_cast<uint32_t>(lane) < S.k)
+            ? reinterpret_cast<unsigned long long>(members[S.member_off + lane].cand) : 0ull;
+        const unsigned long long ref = reinterpret_cast<unsigned long long>(S.ref);
+        for (uint64_t t = t0; t < t1 && !g.dead; ++t) {
+            const unsigned long long off = t * tile_bytes;
+            for (uint32_t j = 0; j <= S.k; ++j) {
+                const unsigned long long base = __shfl_sync(full, mine, j == 0 ? 0 : static_cast<int>(j - 1));
+                const unsigned long long src = (j == 0 ? ref : base) + off;
+                int ok = 1;
+                if (lane == 0) {
+                    ok = mbar_wait(g.empty(), g.phase ^ 1u, g.abort_flag) ? 1 : 0;
+                    if (ok) {
+                        mbar_arrive_expect_tx(g.full(), tile_bytes);
+                        bulk_load(g.data(), reinterpret_cast<const void*>(src), tile_bytes, g.full(), pol);
+                    }
+                }
+                ok = __shfl_sync(full, ok, 0);
+                if (!ok) { g.dead = true; break; }
+                g.advance();
+                ++issued;
+            }
+        }
+    }
+    return issued;
+}
+
+__global__ void __launch_bounds__(kBlock, kCtasPerSm)
 validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
-               const CtaRange* __restrict__ ranges, Acc* __restrict__ partials, float atol, float rtol) {
+               const CtaRange* __restrict__ ranges, Acc* __restrict__ partials, float atol, float rtol,
+               uint32_t* __restrict__ status) {
+    extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ Acc s_acc[kMaxK][kWarps];
     __shared__ const void* s_cand[kMaxK];
+    __shared__ __align__(8) unsigned long long s_full[kStages], s_empty[kStages];
+    __shared__ int s_abort;
     const CtaRange rg = ranges[blockIdx.x];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (uint32_t s = rg.s_begin; s <= rg.s_end && rg.s_begin <= rg.s_end; ++s) {
-        const SetRec S = sets[s];
-        const uint64_t tiles = (S.n + tile_elems(S.dtype) - 1) / tile_elems(S.dtype);
-        const uint64_t t0 = (s == rg.s_begin) ? rg.t_begin : 0;
-        const uint64_t t1 = (s == rg.s_end) ? rg.t_end : tiles;
-        if (t0 >= t1) continue;
-        for (uint32_t i = threadIdx.x; i < S.k * kWarps; i += kThreads) {
-            Acc z;
-            z.mism = 0; z.nonfin = 0; z.sse = 0.0; z.max_abs = 0; z.max_rel = 0; z.flags = 0; z.pad = 0;
-            s_acc[i / kWarps][i % kWarps] = z;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(smem_u32(&s_full[i]), 1);          // the producer's arrive + the copy's bytes
+            mbar_init(smem_u32(&s_empty[i]), kWarps);    // one arrive per consumer warp
         }
-        if (threadIdx.x < S.k) s_cand[threadIdx.x] = members[S.member_off + threadIdx.x].cand;
-        __syncthreads();
-        if (S.dtype == EVO_F32) run_set<EVO_F32>(S, t0, t1, atol, rtol, s_acc, s_cand, warp, lane);
-        else if (S.dtype == EVO_F16) run_set<EVO_F16>(S, t0, t1, atol, rtol, s_acc, s_cand, warp, lane);
-        else run_set<EVO_BF16>(S, t0, t1, atol, rtol, s_acc, s_cand, warp, lane);
-        __syncthreads();
-        if (threadIdx.x < S.k) {
-            Acc a = s_acc[threadIdx.x][0];
-#pragma unroll
-            for (int w = 1; w < kWarps; ++w) {
-                const Acc b = s_acc[threadIdx.x][w];
-                a.mism += b.mism; a.nonfin += b.nonfin; a.sse += b.sse;
-                a.max_abs = max(a.max_abs, b.max_abs); a.max_rel = max(a.max_rel, b.max_rel); a.flags |= b.flags;
+        s_abort = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    Ring g;
+    g.full0 = smem_u32(&s_full[0]);
+    g.empty0 = smem_u32(&s_empty[0]);
+    g.data0 = smem_u32(s_ring);
+    g.abort_flag = &s_abort;
+    uint32_t issued = 0;
+
+    if (warp == kWarps) {
+        issued = producer_loop(sets, members, rg, g, lane);
+    } else {
+        for (uint32_t s = rg.s_begin; s <= rg.s_end; ++s) {
+            const SetRec S = sets[s];
+            uint64_t t0, t1, ring_tiles;
+            set_span(rg, s, S, &t0, &t1, &ring_tiles);
+            if (t0 >= t1) continue;
+            for (uint32_t i = threadIdx.x; i < S.k * kWarps; i += kThreads) {
+                Acc z;
+                z.mism = 0; z.nonfin = 0; z.sse = 0.0; z.max_abs = 0; z.max_rel = 0; z.flags = 0; z.pad = 0;
+                s_acc[i / kWarps][i % kWarps] = z;
             }
-            partials[rg.part_base + (S.member_off - rg.first_member) + threadIdx.x] = a;
+            if (threadIdx.x < S.k) s_cand[threadIdx.x] = members[S.member_off + threadIdx.x].cand;
+            consumer_bar();
+            if (S.dtype == EVO_F32) run_set<EVO_F32>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_cand, g, warp, lane);
+            else if (S.dtype == EVO_F16) run_set<EVO_F16>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_cand, g, warp, lane);
+            else run_set<EVO_BF16>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_cand, g, warp, lane);
+            consumer_bar();
+            if (threadIdx.x < S.k) {
+                Acc a = s_acc[threadIdx.x][0];
+#pragma unroll
+                for (int w = 1; w < kWarps; ++w) {
+                    const Acc b = s_acc[threadIdx.x][w];
+                    a.mism += b.mism; a.nonfin += b.nonfin; a.sse += b.sse;
+                    a.max_abs = max(a.max_abs, b.max_abs); a.max_rel = max(a.max_rel, b.max_rel); a.flags |= b.flags;
+                }
+                partials[rg.part_base + (S.member_off - rg.first_member) + threadIdx.x] = a;
+            }
+            consumer_bar();
         }
-        __syncthreads();
+    }
+    __syncthreads();
+    if (s_abort) {
+        // A wait ran out.  Before the CTA gives its shared memory back, let the copies that
+        // are still outstanding land (bounded again), then report.
+        if (warp == kWarps && lane == 0) {
+            const uint32_t pending = issued < kStages ? issued : kStages;
+            for (uint32_t q = 0; q < pending; ++q) {
+                const uint32_t i = issued - 1 - q;
+                const uint32_t bar = g.full0 + 8u * (i % kStages);
+                const uint32_t parity = (i / kStages) & 1u;
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(bar, parity) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+        if (threadIdx.x == 0) atomicOr(status, 1u);
     }
 }
 
 // One warp per tensor: fold the partial records of the CTAs [cta_first, cta_last] in a
-// fixed order (lane-strided, then a xor tree).
+// fixed order (lane-strided, then a xor tree).  If the first pass gave up on a wait, the
+// records are incomplete: every result then says so instead of carrying numbers.
 __global__ void __launch_bounds__(kThreads)
 validate_pass2(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
                const CtaRange* __restrict__ ranges, const Acc* __restrict__ partials,
-               uint32_t n_members, evo_result* __restrict__ results) {
+               uint32_t n_members, evo_result* __restrict__ results, const uint32_t* __restrict__ status) {
     const uint32_t m = blockIdx.x * kWarps + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (m >= n_members) return;
     const MemberRec M = members[m];
+    if (*status != 0) {
+        if (lane == 0) {
+            evo_result r;
+            r.n_mismatch = 0; r.n_nonfinite = 0; r.sse = 0.0; r.max_abs = 0.f; r.max_rel = 0.f;
+            r.flags = EVO_FLAG_INCOMPLETE; r.pass = 0;
+            results[M.desc] = r;
+        }
+        return;
+    }
     const SetRec S = sets[M.set];
     unsigned long long mism = 0, nonfin = 0;
     double sse = 0.0;
@@ -393,8 +638,14 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     const cudaEvent_t ev_start = ctx->time_start, ev_stop = ctx->time_stop;
     ctx->time_start = ctx->time_stop = nullptr;
     if (ev_start) EVO_CUDA_TRY(ctx, cudaEventRecord(ev_start, stream));
+    uint32_t* d_status = evo::status_word(ctx);
     if (n_ctas > 0) {
-        validate_pass1<<<n_ctas, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol);
+        if (!ctx->pass1_ready) {
+            EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(validate_pass1, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   static_cast<int>(kRingBytes)));
+            ctx->pass1_ready = true;
+        }
+        validate_pass1<<<n_ctas, kBlock, kRingBytes, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol, d_status);
         ctx->launches += 1;
         EVO_CUDA_TRY(ctx, cudaGetLastError());
     }
@@ -402,7 +653,7 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     const uint32_t n_members = static_cast<uint32_t>(n_desc);
     if (n_members > 0) {
         validate_pass2<<<(n_members + kWarps - 1) / kWarps, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts,
-                                                                                    n_members, results);
+                                                                                    n_members, results, d_status);
         ctx->launches += 1;
         EVO_CUDA_TRY(ctx, cudaGetLastError());
     }
@@ -492,8 +743,7 @@ extern "C" int evo_validate_host(evo_ctx* ctx, const void* const* cand_ptrs, con
     if (st != EVO_OK) return st;
     if (n_desc) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(results, d_results, n_desc * sizeof(evo_result), cudaMemcpyDeviceToHost, stream));
     if (group_pass) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(group_pass, d_gpass, n_group * sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
-    EVO_CUDA_TRY(ctx, cudaStreamSynchronize(stream));
-    return EVO_OK;
+    return evo::sync_and_check(ctx, stream, who);
 }
 
 // ---- evo_validate_static: the same check without any allocation --------------------------
@@ -508,6 +758,7 @@ namespace {
 
 constexpr int kMaxDevices = 64;
 struct StaticDevice { unsigned char* scratch; int sm_count; bool ready; };
+constexpr size_t kStaticStatusBytes = 256;      // the scratch starts with the status word (zero when the library loads)
 StaticDevice g_static_dev[kMaxDevices];
 std::mutex g_static_mutex;
 thread_local char g_static_error[256] = "";
@@ -547,6 +798,8 @@ extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref
             int sms = 0;
             e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
             if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: %s", cudaGetErrorString(e));
+            e = cudaFuncSetAttribute(validate_pass1, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kRingBytes));
+            if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: %s", cudaGetErrorString(e));
             g_static_dev[device].scratch = ptr;
             g_static_dev[device].sm_count = sms;
             g_static_dev[device].ready = true;
@@ -561,8 +814,8 @@ extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref
                               &plan, &err);
     if (st != EVO_OK) return static_fail(st, "evo_validate_static: %s", err.c_str());
 
-    // Layout inside the scratch: the plan, then the partial records.
-    const size_t o_sets = 0;
+    // Layout inside the scratch: the status word, the plan, then the partial records.
+    const size_t o_sets = kStaticStatusBytes;
     const size_t o_members = align_up(o_sets + plan.sets.size() * sizeof(SetRec), 256);
     const size_t o_ranges = align_up(o_members + plan.members.size() * sizeof(MemberRec), 256);
     const size_t o_goff = align_up(o_ranges + plan.ranges.size() * sizeof(CtaRange), 256);
@@ -578,15 +831,16 @@ extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref
 
     // The plan goes up from ordinary host memory: the copy call returns once the runtime has
     // taken the bytes, so the local buffer may go out of scope.
-    std::vector<unsigned char> h(plan_bytes ? plan_bytes : 1);
-    auto put = [&](size_t o, const void* src, size_t bytes) { if (bytes) std::memcpy(h.data() + o, src, bytes); };
+    const size_t up_bytes = plan_bytes - kStaticStatusBytes;
+    std::vector<unsigned char> h(up_bytes ? up_bytes : 1);
+    auto put = [&](size_t o, const void* src, size_t bytes) { if (bytes) std::memcpy(h.data() + (o - kStaticStatusBytes), src, bytes); };
     put(o_sets, plan.sets.data(), plan.sets.size() * sizeof(SetRec));
     put(o_members, plan.members.data(), plan.members.size() * sizeof(MemberRec));
     put(o_ranges, plan.ranges.data(), plan.ranges.size() * sizeof(CtaRange));
     put(o_goff, plan.group_off.data(), plan.group_off.size() * 4);
     put(o_gdesc, plan.group_desc.data(), plan.group_desc.size() * 4);
-    if (plan_bytes) {
-        e = cudaMemcpyAsync(dev.scratch, h.data(), plan_bytes, cudaMemcpyHostToDevice, stream);
+    if (up_bytes) {
+        e = cudaMemcpyAsync(dev.scratch + kStaticStatusBytes, h.data(), up_bytes, cudaMemcpyHostToDevice, stream);
         if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: plan upload: %s", cudaGetErrorString(e));
     }
     const unsigned char* d = dev.scratch;
@@ -594,14 +848,19 @@ extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref
     const MemberRec* d_members = reinterpret_cast<const MemberRec*>(d + o_members);
     const CtaRange* d_ranges = reinterpret_cast<const CtaRange*>(d + o_ranges);
     Acc* d_parts = reinterpret_cast<Acc*>(dev.scratch + o_parts);
-    // Nothing in the scratch has to start at zero: pass 1 writes every partial record that
-    // pass 2 reads, so what an earlier call left behind is never looked at.
+    // Nothing in the plan or the partial records has to start at zero: pass 1 writes every
+    // record that pass 2 reads, so what an earlier call left behind is never looked at.  The
+    // status word is zero from the library image and is only ever raised (a wait that ran out
+    // in pass 1); it is deliberately not cleared, so that such a failure stays visible: every
+    // later call on this device then reports incomplete results.
+    uint32_t* d_status = reinterpret_cast<uint32_t*>(dev.scratch);
     const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
-    if (n_ctas > 0) validate_pass1<<<n_ctas, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol);
+    if (n_ctas > 0)
+        validate_pass1<<<n_ctas, kBlock, kRingBytes, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol, d_status);
     const uint32_t n_members = static_cast<uint32_t>(n_desc);
     if (n_members > 0)
         validate_pass2<<<(n_members + kWarps - 1) / kWarps, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts,
-                                                                                    n_members, results);
+                                                                                    n_members, results, d_status);
     if (group_pass)
         group_verdict<<<static_cast<unsigned>((n_group + 255) / 256), 256, 0, stream>>>(
             reinterpret_cast<const uint32_t*>(d + o_goff), reinterpret_cast<const uint32_t*>(d + o_gdesc), results,

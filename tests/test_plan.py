@@ -7,7 +7,7 @@ import pytest
 
 DESC = np.dtype([("n", "<u8"), ("ref", "<u8"), ("dtype", "<i4"), ("group", "<u4")], align=True)
 RANGE = np.dtype([("tile_begin", "<u8"), ("tile_end", "<u8"), ("set_begin", "<u4"), ("set_end", "<u4")], align=True)
-SUMMARY = np.dtype([("n_sets", "<u4"), ("n_ctas", "<u4"), ("n_parts", "<u4"), ("tile_bytes", "<u4"), ("total_tiles", "<u8")], align=True)
+SUMMARY = np.dtype([("n_sets", "<u4"), ("n_ctas", "<u4"), ("n_parts", "<u4"), ("tile_elems", "<u4"), ("total_tiles", "<u8")], align=True)
 F32, F16, BF16 = 1, 2, 3
 ESIZE = {F32: 4, F16: 2, BF16: 2}
 
@@ -63,8 +63,8 @@ def coverage(summ, ranges, set_tiles):
     return weights
 
 
-def tiles_of(n, dtype, tile_bytes):
-    per = tile_bytes // ESIZE[dtype]
+def tiles_of(n, dtype, tile_elems):
+    per = tile_elems
     return (n + per - 1) // per
 
 
@@ -75,7 +75,7 @@ def test_shared_reference_becomes_one_set_and_cut_is_balanced(lib):
     cands = 0x1000_0000_0000 + np.arange(16, dtype=np.uint64) * (n * 4)
     st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
     assert st == 0 and summ["n_sets"] == 1 and set_k.tolist() == [16] and set(set_of.tolist()) == {0}
-    tiles = tiles_of(n, F32, int(summ["tile_bytes"]))
+    tiles = tiles_of(n, F32, int(summ["tile_elems"]))
     assert summ["total_tiles"] == tiles and summ["n_ctas"] == 444 and tiles > 444
     w = coverage(summ, ranges, [tiles])
     assert max(w) - min(w) <= 1
@@ -89,7 +89,7 @@ def test_more_members_than_a_set_holds(lib):
     st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 64)
     assert st == 0 and set_k.tolist() == [32, 32, 32, 4]
     assert set_of.tolist() == [i // 32 for i in range(100)]
-    tiles = tiles_of(50000, BF16, int(summ["tile_bytes"]))
+    tiles = tiles_of(50000, BF16, int(summ["tile_elems"]))
     coverage(summ, ranges, [tiles] * 4)
 
 
@@ -108,7 +108,7 @@ def test_ragged_mixed_population(lib):
     for max_ctas in (1, 7, 148 * 3, 5000):
         st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, max_ctas)
         assert st == 0
-        tb = int(summ["tile_bytes"])
+        tb = int(summ["tile_elems"])
         set_tiles = [None] * int(summ["n_sets"])
         weight_per_tile = [None] * int(summ["n_sets"])
         for i in range(n_desc):
@@ -139,7 +139,7 @@ def test_ragged_mixed_population(lib):
 def test_heavy_items_with_few_tiles_leave_no_idle_cta(lib):
     # 40 members of 3 tiles each: 12 items of very different weight, fewer runs than items
     descs = np.zeros(80, DESC)
-    descs["n"], descs["dtype"] = 20000, F16
+    descs["n"], descs["dtype"] = 10000, F16
     descs["ref"][:40], descs["ref"][40:] = 0x7000_0000_0000, 0x7100_0000_0000
     cands = 0x1000_0000_0000 + np.arange(80, dtype=np.uint64) * 65536
     st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
@@ -181,4 +181,4 @@ def test_unaligned_tensors_are_scheduled_too(lib):
     descs["n"], descs["ref"], descs["dtype"] = 100000, 0x7000_0000_0004, F32
     st, summ, ranges, set_of, set_k = inspect(lib, [0x1000_0000, 0x2000_0008], descs, 16)
     assert st == 0 and summ["n_sets"] == 1
-    coverage(summ, ranges, [tiles_of(100000, F32, int(summ["tile_bytes"]))])
+    coverage(summ, ranges, [tiles_of(100000, F32, int(summ["tile_elems"]))])
