@@ -108,6 +108,12 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 
+__device__ __forceinline__ float rcp_approx(float x) {
+    float y;
+    asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -268,8 +274,8 @@ constexpr float kShrink = 0.99999904632568359375f;      // 1 - 2^-20
 // filter fired walks its 16 elements again in registers and divides only where r != 0 and
 // the filter still fires against its own, rising maximum.
 template <int DT>
-__device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float atol, float rtol,
-                                          Acc (*s_acc)[kWarps], const void* const* s_cand, Ring& g, int warp, int lane) {
+__device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float atol, float rtol, Acc (*s_acc)[kWarps],
+                                          uint32_t* s_mr, const void* const* s_cand, Ring& g, int warp, int lane) {
     using E = Elem<DT>;
     if (g.dead) return;
     constexpr uint32_t kVecStride = kThreads * 16;
@@ -300,7 +306,9 @@ __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float ato
         }
         ring_release(g, lane);
         Acc* acc = &s_acc[k][warp];
-        const float m = __uint_as_float(acc->max_rel);
+        // Running maximum of d/|r| of this member, shared by the CTA's warps.  A stale (smaller)
+        // value only makes the filter fire more often.
+        const float m = __uint_as_float(*reinterpret_cast<volatile uint32_t*>(&s_mr[k]));
         const float mlo = __fmul_rz(m, kShrink);
         uint32_t cnt = 0;
         float ma = 0.f, sse = 0.f;
@@ -320,8 +328,35 @@ __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float ato
         // squares is then NaN/Inf) or if every d is so small that d^2 underflows in binary32.
         const bool redo = !(sse < kInf) || (ma < 9.094947017729282e-13f /* 2^-40 */ && ma > 0.f);
         float mt = m;
-        if (trig && !redo) {
-            float lo = mlo;
+        float lo = mlo;
+        bool scan = trig && !redo;
+        const unsigned full = 0xffffffffu;
+        if (m == 0.f && __any_sync(full, scan)) {
+            // No maximum yet (m is the same for the whole warp): every lane with some d > 0 would
+            // scan, each dividing at its own elements.  Instead all lanes first form approximate
+            // quotients (reciprocal approximation, relative error below 2^-21), the warp takes
+            // their maximum A, and only lanes that come within 2^-17 of A scan, starting from a
+            // threshold 2^-18 below A: the element with the exact maximum passes it.
+            float qa = 0.f;
+            if (!redo) {
+#pragma unroll
+                for (int v = 0; v < E::kVecs; ++v)
+#pragma unroll
+                    for (int e = 0; e < E::kPerVec; ++e) {
+                        const int i = v * E::kPerVec + e;
+                        const float ar = fabsf(r[i]);
+                        const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
+                        qa = fmaxf(qa, d * rcp_approx(ar == 0.f ? kInf : ar));      // r == 0 contributes 0
+                    }
+            }
+            const float A = __uint_as_float(__reduce_max_sync(full, __float_as_uint(qa)));
+            // Outside the range where the error bound of the approximation holds, scan from 0.
+            if (A > 7.888609052210118e-31f /* 2^-100 */ && A < kInf) {
+                lo = __fmul_rz(A, 0.999996185302734375f /* 1 - 2^-18 */);
+                scan = scan && qa >= __fmul_rz(A, 0.99999237060546875f /* 1 - 2^-17 */);
+            }
+        }
+        if (scan) {
 #pragma unroll
             for (int v = 0; v < E::kVecs; ++v)
 #pragma unroll
@@ -335,7 +370,6 @@ __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float ato
                     }
                 }
         }
-        const unsigned full = 0xffffffffu;
         if (__any_sync(full, redo)) {
             Lane st;
             if (redo) {
@@ -344,6 +378,8 @@ __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float ato
             } else {
                 st.cnt = cnt; st.ma = ma; st.mr = mt; st.dsse = static_cast<double>(sse);
             }
+            const uint32_t mr_w = __reduce_max_sync(full, __float_as_uint(st.mr));
+            if (lane == 0 && mr_w > __float_as_uint(m)) atomicMax(&s_mr[k], mr_w);
             warp_commit_exact(st, acc, lane);
         } else {
             const uint32_t cnt_w = __reduce_add_sync(full, cnt);
@@ -356,9 +392,8 @@ __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float ato
                 acc->mism += cnt_w;
                 acc->sse += static_cast<double>(x);
                 acc->max_abs = max(acc->max_abs, ma_w);
-                acc->max_rel = max(acc->max_rel, mr_w);
+                if (mr_w > __float_as_uint(m)) atomicMax(&s_mr[k], mr_w);
             }
-            __syncwarp();
         }
     }
 }
@@ -393,9 +428,9 @@ __device__ __forceinline__ void set_span(const CtaRange& rg, uint32_t s, const S
 
 template <int DT>
 __device__ __forceinline__ void run_set(const SetRec& S, uint64_t t0, uint64_t t1, uint64_t ring_tiles, float atol, float rtol,
-                                        Acc (*s_acc)[kWarps], const void* const* s_cand, Ring& g, int warp, int lane) {
+                                        Acc (*s_acc)[kWarps], uint32_t* s_mr, const void* const* s_cand, Ring& g, int warp, int lane) {
     for (uint64_t t = t0; t < t1; ++t) {
-        if (t < ring_tiles) fast_tile<DT>(S, t, atol, rtol, s_acc, s_cand, g, warp, lane);
+        if (t < ring_tiles) fast_tile<DT>(S, t, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
         else if (!g.dead) slow_tile<DT>(S, t, atol, rtol, s_acc, s_cand, warp, lane);
     }
 }
@@ -450,6 +485,7 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ Acc s_acc[kMaxK][kWarps];
     __shared__ const void* s_cand[kMaxK];
+    __shared__ uint32_t s_mr[kMaxK];         // per member: running maximum of d/|r| found on the fast path (bit pattern)
     __shared__ __align__(8) unsigned long long s_full[kStages], s_empty[kStages];
     __shared__ int s_abort;
     const CtaRange rg = ranges[blockIdx.x];
@@ -483,11 +519,14 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
                 z.mism = 0; z.nonfin = 0; z.sse = 0.0; z.max_abs = 0; z.max_rel = 0; z.flags = 0; z.pad = 0;
                 s_acc[i / kWarps][i % kWarps] = z;
             }
-            if (threadIdx.x < S.k) s_cand[threadIdx.x] = members[S.member_off + threadIdx.x].cand;
+            if (threadIdx.x < S.k) {
+                s_cand[threadIdx.x] = members[S.member_off + threadIdx.x].cand;
+                s_mr[threadIdx.x] = 0;
+            }
             consumer_bar();
-            if (S.dtype == EVO_F32) run_set<EVO_F32>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_cand, g, warp, lane);
-            else if (S.dtype == EVO_F16) run_set<EVO_F16>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_cand, g, warp, lane);
-            else run_set<EVO_BF16>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_cand, g, warp, lane);
+            if (S.dtype == EVO_F32) run_set<EVO_F32>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
+            else if (S.dtype == EVO_F16) run_set<EVO_F16>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
+            else run_set<EVO_BF16>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
             consumer_bar();
             if (threadIdx.x < S.k) {
                 Acc a = s_acc[threadIdx.x][0];
@@ -497,6 +536,7 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
                     a.mism += b.mism; a.nonfin += b.nonfin; a.sse += b.sse;
                     a.max_abs = max(a.max_abs, b.max_abs); a.max_rel = max(a.max_rel, b.max_rel); a.flags |= b.flags;
                 }
+                a.max_rel = max(a.max_rel, s_mr[threadIdx.x]);
                 partials[rg.part_base + (S.member_off - rg.first_member) + threadIdx.x] = a;
             }
             consumer_bar();
