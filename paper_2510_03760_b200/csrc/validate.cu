@@ -274,7 +274,7 @@ constexpr float kShrink = 0.99999904632568359375f;      // 1 - 2^-20
 // filter fired walks its 16 elements again in registers and divides only where r != 0 and
 // the filter still fires against its own, rising maximum.
 template <int DT>
-__device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float atol, float rtol, Acc (*s_acc)[kWarps],
+__device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, float atol, float rtol, Acc (*s_acc)[kWarps],
                                           uint32_t* s_mr, const void* const* s_cand, Ring& g, int warp, int lane) {
     using E = Elem<DT>;
     if (g.dead) return;
@@ -294,7 +294,6 @@ __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float ato
 #pragma unroll
     for (int e = 0; e < kEpt; ++e) tol[e] = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r[e])));
     const uint64_t vec0 = t * (kTileElems / E::kPerVec) + threadIdx.x;   // this thread's first vector of the tile
-    const int K = static_cast<int>(S.k);
 #pragma unroll 1
     for (int k = 0; k < K; ++k) {
         if (!ring_acquire(g)) return;
@@ -373,7 +372,7 @@ __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float ato
         if (__any_sync(full, redo)) {
             Lane st;
             if (redo) {
-                exact_redo<DT>(static_cast<const uint4*>(s_cand[k]) + vec0, static_cast<const uint4*>(S.ref) + vec0,
+                exact_redo<DT>(static_cast<const uint4*>(s_cand[k]) + vec0, static_cast<const uint4*>(ref) + vec0,
                                atol, rtol, &st);
             } else {
                 st.cnt = cnt; st.ma = ma; st.mr = mt; st.dsse = static_cast<double>(sse);
@@ -398,8 +397,8 @@ __device__ __forceinline__ void fast_tile(const SetRec& S, uint64_t t, float ato
     }
 }
 
-// Ragged last tile, or tensors that are not 16-byte aligned: scalar loads straight from
-// global memory, exact rule.  These tiles do not pass through the ring.
+// Tensors that are not 16-byte aligned: scalar loads straight from global memory, exact
+// rule.  These tiles do not pass through the ring.
 template <int DT>
 __device__ __noinline__ void slow_tile(const SetRec& S, uint64_t t, float atol, float rtol,
                                        Acc (*s_acc)[kWarps], const void* const* s_cand, int warp, int lane) {
@@ -416,22 +415,135 @@ __device__ __noinline__ void slow_tile(const SetRec& S, uint64_t t, float atol, 
     }
 }
 
-// Tiles of set s that belong to this CTA's range, and how many of the set's tiles are full
-// and aligned (those travel through the ring; producer and consumers must agree on this).
-__device__ __forceinline__ void set_span(const CtaRange& rg, uint32_t s, const SetRec& S, uint64_t* t0, uint64_t* t1,
-                                         uint64_t* ring_tiles) {
+// The ragged last tile of an aligned tensor.  Its whole 16-byte vectors (`valid_vecs` of
+// them) come through the ring like a full tile; a thread takes the same vectors as in
+// fast_tile but only those that exist, and applies the exact rule to each element.  Once per
+// tensor, so kept out of line and simple.
+// The ring position travels by value (in and out, packed), so that the caller's copy can
+// stay in registers.
+template <int DT>
+__device__ __noinline__ uint32_t tail_tile(uint32_t n_members, uint32_t valid_vecs, float atol, float rtol,
+                                           Acc (*s_acc)[kWarps], Ring g, int warp, int lane) {
+    using E = Elem<DT>;
+    constexpr uint32_t kVecStride = kThreads * 16;
+    uint4 rv[E::kVecs];
+    if (ring_acquire(g)) {
+        const uint32_t a = g.data() + threadIdx.x * 16;
+#pragma unroll
+        for (int v = 0; v < E::kVecs; ++v) rv[v] = lds128(a + v * kVecStride);
+        ring_release(g, lane);
+        for (uint32_t k = 0; k < n_members; ++k) {
+            if (!ring_acquire(g)) break;
+            uint4 cv[E::kVecs];
+            const uint32_t b = g.data() + threadIdx.x * 16;
+#pragma unroll
+            for (int v = 0; v < E::kVecs; ++v) cv[v] = lds128(b + v * kVecStride);
+            ring_release(g, lane);
+            Lane st;
+#pragma unroll
+            for (int v = 0; v < E::kVecs; ++v) {
+                if (v * kThreads + threadIdx.x < valid_vecs) {
+#pragma unroll
+                    for (int e = 0; e < E::kPerVec; ++e) exact_elem(E::at(cv[v], e), E::at(rv[v], e), atol, rtol, st);
+                }
+            }
+            warp_commit_exact(st, &s_acc[k][warp], lane);
+        }
+    }
+    return g.stage | (g.phase << 8) | (g.dead ? 1u << 16 : 0u);       // ring_pack
+}
+
+// The last few elements of an aligned tensor that do not fill a 16-byte vector (at most 3
+// fp32 or 7 fp16/bf16 values): thread (8k + j) takes element j of member k, so one round of
+// scalar loads serves all members; groups of 8 lanes fold with shuffles and the group's first
+// lane adds to the accumulator its own warp owns.
+template <int DT>
+__device__ __noinline__ void leftover_pass(const SetRec& S, uint64_t e_first, uint32_t left, float atol, float rtol,
+                                           Acc (*s_acc)[kWarps], const void* const* s_cand, int warp, int lane) {
+    using E = Elem<DT>;
+    using T = typename E::T;
+    const uint32_t k = threadIdx.x >> 3, j = threadIdx.x & 7;
+    Lane st;
+    if (k < S.k && j < left) {
+        const T c = static_cast<const T*>(s_cand[k])[e_first + j];
+        const T r = static_cast<const T*>(S.ref)[e_first + j];
+        exact_elem(E::widen(c), E::widen(r), atol, rtol, st);
+    }
+    const unsigned full = 0xffffffffu;
+#pragma unroll
+    for (int o = 4; o > 0; o >>= 1) {
+        st.cnt += __shfl_xor_sync(full, st.cnt, o);
+        st.nf += __shfl_xor_sync(full, st.nf, o);
+        st.flags |= __shfl_xor_sync(full, st.flags, o);
+        st.ma = fmaxf(st.ma, __shfl_xor_sync(full, st.ma, o));
+        st.mr = fmaxf(st.mr, __shfl_xor_sync(full, st.mr, o));
+        st.dsse += __shfl_xor_sync(full, st.dsse, o);
+    }
+    if (j == 0 && k < S.k) {
+        Acc* acc = &s_acc[k][warp];                 // warp == k / 4: touched by this warp only
+        acc->mism += st.cnt;
+        acc->nonfin += st.nf;
+        acc->sse += st.dsse;
+        acc->max_abs = max(acc->max_abs, __float_as_uint(st.ma));
+        acc->max_rel = max(acc->max_rel, __float_as_uint(st.mr));
+        acc->flags |= st.flags;
+    }
+    __syncwarp();
+}
+
+// What of set s belongs to this CTA's range, and how its tiles travel.  Producer and
+// consumers derive the sequence of ring stages from this, so they must agree on it.
+struct Span {
+    uint64_t t0, t1;         // this CTA's tiles of the set
+    uint64_t full_tiles;     // tiles [0, full_tiles) are complete and go through the ring (0 if not 16-byte aligned)
+    uint32_t tail_vecs;      // whole 16-byte vectors of the ragged last tile, copied through the ring as well
+    uint32_t left;           // elements after those (less than one vector): leftover pass
+};
+__device__ __forceinline__ Span set_span(const CtaRange& rg, uint32_t s, const SetRec& S) {
+    Span sp;
     const uint64_t tiles = (S.n + kTileElems - 1) / kTileElems;
-    *t0 = (s == rg.s_begin) ? rg.t_begin : 0;
-    *t1 = (s == rg.s_end) ? rg.t_end : tiles;
-    *ring_tiles = S.vec_ok ? S.n / kTileElems : 0;
+    sp.t0 = (s == rg.s_begin) ? rg.t_begin : 0;
+    sp.t1 = (s == rg.s_end) ? rg.t_end : tiles;
+    const uint32_t rem = static_cast<uint32_t>(S.n % kTileElems);
+    const uint32_t per_vec = S.dtype == EVO_F32 ? 4u : 8u;
+    sp.full_tiles = S.vec_ok ? S.n / kTileElems : 0;
+    sp.tail_vecs = S.vec_ok ? rem / per_vec : 0;
+    sp.left = S.vec_ok ? rem % per_vec : 0;
+    return sp;
+}
+
+// All full tiles [t_begin, t_end) of a set: the hot loop, a function of its own so that its
+// registers are allocated without regard to the rarely used paths around it.  The ring
+// position travels by value, in and packed out.
+__device__ __forceinline__ uint32_t ring_pack(const Ring& g) { return g.stage | (g.phase << 8) | (g.dead ? 1u << 16 : 0u); }
+__device__ __forceinline__ void ring_unpack(Ring& g, uint32_t pos) {
+    g.stage = pos & 0xffu; g.phase = (pos >> 8) & 1u; g.dead = (pos >> 16) != 0;
+}
+template <int DT>
+__device__ __noinline__ uint32_t fast_run(const void* ref, int K, uint64_t t_begin, uint64_t t_end, float atol, float rtol,
+                                          Acc (*s_acc)[kWarps], uint32_t* s_mr, const void* const* s_cand, Ring g,
+                                          int warp, int lane) {
+#pragma unroll 1
+    for (uint64_t t = t_begin; t < t_end; ++t) fast_tile<DT>(ref, K, t, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
+    return ring_pack(g);
 }
 
 template <int DT>
-__device__ __forceinline__ void run_set(const SetRec& S, uint64_t t0, uint64_t t1, uint64_t ring_tiles, float atol, float rtol,
-                                        Acc (*s_acc)[kWarps], uint32_t* s_mr, const void* const* s_cand, Ring& g, int warp, int lane) {
-    for (uint64_t t = t0; t < t1; ++t) {
-        if (t < ring_tiles) fast_tile<DT>(S, t, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
-        else if (!g.dead) slow_tile<DT>(S, t, atol, rtol, s_acc, s_cand, warp, lane);
+__device__ __forceinline__ void run_set(const SetRec& S, const Span& sp, float atol, float rtol, Acc (*s_acc)[kWarps],
+                                        uint32_t* s_mr, const void* const* s_cand, Ring& g, int warp, int lane) {
+    using E = Elem<DT>;
+    if (!S.vec_ok) {
+        for (uint64_t t = sp.t0; t < sp.t1; ++t) slow_tile<DT>(S, t, atol, rtol, s_acc, s_cand, warp, lane);
+        return;
+    }
+    const uint64_t t_full = sp.t1 < sp.full_tiles ? sp.t1 : sp.full_tiles;
+    if (sp.t0 < t_full)
+        ring_unpack(g, fast_run<DT>(S.ref, static_cast<int>(S.k), sp.t0, t_full, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane));
+    if (sp.t1 > sp.full_tiles) {        // the ragged last tile is in this CTA's range
+        if (sp.tail_vecs && !g.dead) ring_unpack(g, tail_tile<DT>(S.k, sp.tail_vecs, atol, rtol, s_acc, g, warp, lane));
+        if (sp.left && !g.dead)
+            leftover_pass<DT>(S, sp.full_tiles * kTileElems + static_cast<uint64_t>(sp.tail_vecs) * E::kPerVec, sp.left,
+                              atol, rtol, s_acc, s_cand, warp, lane);
     }
 }
 
@@ -447,16 +559,17 @@ __device__ __forceinline__ uint32_t producer_loop(const SetRec* __restrict__ set
     uint32_t issued = 0;
     for (uint32_t s = rg.s_begin; s <= rg.s_end && !g.dead; ++s) {
         const SetRec S = sets[s];
-        uint64_t t0, t1, ring_tiles;
-        set_span(rg, s, S, &t0, &t1, &ring_tiles);
-        if (t1 > ring_tiles) t1 = ring_tiles;
+        const Span sp = set_span(rg, s, S);
+        const uint64_t ring_end = sp.full_tiles + (sp.tail_vecs ? 1 : 0);     // tiles [0, ring_end) use the ring
+        const uint64_t t0 = sp.t0, t1 = sp.t1 < ring_end ? sp.t1 : ring_end;
         if (t0 >= t1) continue;
-        const uint32_t tile_bytes = kTileElems * (S.dtype == EVO_F32 ? 4u : 2u);
+        const uint32_t full_bytes = kTileElems * (S.dtype == EVO_F32 ? 4u : 2u);
         const unsigned long long mine = (static_cast<uint32_t>(lane) < S.k)
             ? reinterpret_cast<unsigned long long>(members[S.member_off + lane].cand) : 0ull;
         const unsigned long long ref = reinterpret_cast<unsigned long long>(S.ref);
         for (uint64_t t = t0; t < t1 && !g.dead; ++t) {
-            const unsigned long long off = t * tile_bytes;
+            const unsigned long long off = t * full_bytes;
+            const uint32_t tile_bytes = t < sp.full_tiles ? full_bytes : sp.tail_vecs * 16u;
             for (uint32_t j = 0; j <= S.k; ++j) {
                 const unsigned long long base = __shfl_sync(full, mine, j == 0 ? 0 : static_cast<int>(j - 1));
                 const unsigned long long src = (j == 0 ? ref : base) + off;
@@ -511,9 +624,8 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
     } else {
         for (uint32_t s = rg.s_begin; s <= rg.s_end; ++s) {
             const SetRec S = sets[s];
-            uint64_t t0, t1, ring_tiles;
-            set_span(rg, s, S, &t0, &t1, &ring_tiles);
-            if (t0 >= t1) continue;
+            const Span sp = set_span(rg, s, S);
+            if (sp.t0 >= sp.t1) continue;
             for (uint32_t i = threadIdx.x; i < S.k * kWarps; i += kThreads) {
                 Acc z;
                 z.mism = 0; z.nonfin = 0; z.sse = 0.0; z.max_abs = 0; z.max_rel = 0; z.flags = 0; z.pad = 0;
@@ -524,9 +636,9 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
                 s_mr[threadIdx.x] = 0;
             }
             consumer_bar();
-            if (S.dtype == EVO_F32) run_set<EVO_F32>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
-            else if (S.dtype == EVO_F16) run_set<EVO_F16>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
-            else run_set<EVO_BF16>(S, t0, t1, ring_tiles, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
+            if (S.dtype == EVO_F32) run_set<EVO_F32>(S, sp, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
+            else if (S.dtype == EVO_F16) run_set<EVO_F16>(S, sp, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
+            else run_set<EVO_BF16>(S, sp, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
             consumer_bar();
             if (threadIdx.x < S.k) {
                 Acc a = s_acc[threadIdx.x][0];

@@ -131,6 +131,26 @@ def test_unaligned_views_and_ragged_sizes(evo):
                 assert_results_equal(evo.results_to_numpy(res), np.array([want]), "n=%d offs=%d,%d dt=%d" % (n, ro, co, dtype))
 
 
+def test_ragged_tail_of_a_shared_reference_with_specials(evo):
+    # several members per reference (also more than one set holds), a last tile that is ragged
+    # down to a few elements past a 16-byte vector, and NaN/Inf planted in that tail
+    g = torch.Generator().manual_seed(17)
+    for tdt, dtype in [(torch.float32, workloads.F32), (torch.float16, workloads.F16), (torch.bfloat16, workloads.BF16)]:
+        for n, k in [(3 * 4096 + 8 * 5 + 3, 5), (4096 + 7, 34), (2, 3), (9, 1), (2 * 4096 + 16, 2)]:
+            ref = torch.randn(n, generator=g).to(tdt)
+            tensors = []
+            for i in range(k):
+                c = (ref.float() + 0.004 * torch.randn(n, generator=g)).to(tdt)
+                if i % 2 == 0:
+                    c[n - 1] = float("nan")
+                if i % 3 == 0 and n > 12:
+                    c[n - 12] = float("inf")
+                tensors.append(workloads.Tensor(c, 0, i, dtype))
+            pop = workloads.Population("tail n=%d k=%d dt=%d" % (n, k, dtype), [ref], tensors, k, 0.005, 0.005,
+                                       torch.ones(k, 1), torch.ones(1))
+            check(evo, pop)
+
+
 def test_edge_populations(evo):
     g = torch.Generator().manual_seed(11)
     n = 5 * 4096 + 77
