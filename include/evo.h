@@ -278,6 +278,16 @@ EVO_API int evo_set_timing_events(evo_ctx* ctx, void* start, void* stop);
  */
 EVO_API int evo_check(evo_ctx* ctx, void* stream);
 
+/*
+ * evo_selftest_wait - exercise the bounded device-side wait without any fault: enqueues a
+ * one-warp kernel that waits, through the routine the checking kernel uses, on a barrier that
+ * nothing completes, with a limit of `limit_us` microseconds (1..1000000).  The kernel gives
+ * up at the limit, raises the context's status word and returns normally; the next evo_check
+ * then reports EVO_ERR_TIMEOUT once and the context stays usable.  (The paper has no
+ * counterpart.)  Errors: EVO_ERR_ARG, EVO_ERR_CUDA.
+ */
+EVO_API int evo_selftest_wait(evo_ctx* ctx, uint32_t limit_us, void* stream);
+
 /* Number of kernels this context has launched so far (for accounting in benchmarks). */
 EVO_API uint64_t evo_launch_count(const evo_ctx* ctx);
 

@@ -7,6 +7,7 @@ import numpy as np
 import torch
 
 EVO_U32, EVO_F32, EVO_F16, EVO_BF16 = 0, 1, 2, 3
+EVO_FLAG_INCOMPLETE = 0x40000000
 _TORCH_TO_CODE = {torch.float32: EVO_F32, torch.float16: EVO_F16, torch.bfloat16: EVO_BF16}
 
 RESULT_DTYPE = np.dtype(
@@ -50,6 +51,8 @@ def load_library():
     L.evo_set_timing_events.restype = i32
     L.evo_check.argtypes = [vp, vp]
     L.evo_check.restype = i32
+    L.evo_selftest_wait.argtypes = [vp, u32, vp]
+    L.evo_selftest_wait.restype = i32
     L.evo_gen_inputs.argtypes = [vp, u64, u64, i32, u64, vp, vp]
     L.evo_gen_inputs.restype = i32
     for name in ("evo_validate", "evo_validate_host"):
@@ -101,6 +104,10 @@ class Context:
     def synchronize(self, stream=None):
         """evo_check: wait for `stream` and raise EvoError(-6) if a device-side wait ran out."""
         self.check(load_library().evo_check(self._h, _stream_ptr(stream, torch.device("cuda", self.device))))
+
+    def selftest_wait(self, limit_us=1000, stream=None):
+        """evo_selftest_wait: enqueue a kernel whose bounded wait must run out (no fault)."""
+        self.check(load_library().evo_selftest_wait(self._h, int(limit_us), _stream_ptr(stream, torch.device("cuda", self.device))))
 
     def close(self):
         if self._h is not None and _lib is not None:

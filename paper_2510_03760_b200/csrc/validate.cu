@@ -82,17 +82,19 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait, cold part: polls until the phase completes, another warp of the CTA has given
 // up, or the limit has passed (then raises the CTA's abort flag itself).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            unsigned long long limit_ns) {
     const unsigned long long t0 = global_ns();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+        if (global_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag);
+    return mbar_wait_slow(bar, parity, abort_flag, limit_ns);
 }
 __device__ __forceinline__ unsigned long long policy_evict_first() {
     unsigned long long pol;
@@ -733,6 +735,24 @@ __global__ void group_verdict(const uint32_t* __restrict__ offsets, const uint32
     group_pass[g] = ok;
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing will ever complete,
+// through the same wait routine as the first pass, with a short limit; it must come back,
+// raise the status word and leave the context usable.
+__global__ void wait_selftest_kernel(unsigned long long limit_ns, uint32_t* __restrict__ status) {
+    __shared__ __align__(8) unsigned long long s_bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&s_bar), 1);
+        s_abort = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(smem_u32(&s_bar), 0, &s_abort, limit_ns);
+    const bool all_ok = __all_sync(0xffffffffu, ok);
+    __syncthreads();
+    if (threadIdx.x == 0 && (!all_ok || s_abort)) atomicOr(status, 2u);
+}
+
 // ---- host side ------------------------------------------------------------------------
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -896,6 +916,17 @@ extern "C" int evo_validate_host(evo_ctx* ctx, const void* const* cand_ptrs, con
     if (n_desc) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(results, d_results, n_desc * sizeof(evo_result), cudaMemcpyDeviceToHost, stream));
     if (group_pass) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(group_pass, d_gpass, n_group * sizeof(uint32_t), cudaMemcpyDeviceToHost, stream));
     return evo::sync_and_check(ctx, stream, who);
+}
+
+extern "C" int evo_selftest_wait(evo_ctx* ctx, uint32_t limit_us, void* stream) {
+    if (!ctx) return EVO_ERR_ARG;
+    if (limit_us == 0 || limit_us > 1000000u) return evo::fail(ctx, EVO_ERR_ARG, "evo_selftest_wait: limit must be 1..1000000 us");
+    evo::DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
+    wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(1000ull * limit_us, evo::status_word(ctx));
+    ctx->launches += 1;
+    EVO_CUDA_TRY(ctx, cudaGetLastError());
+    return EVO_OK;
 }
 
 // ---- evo_validate_static: the same check without any allocation --------------------------
