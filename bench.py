@@ -60,6 +60,27 @@ def measured_peak():
         return 6650.0, "fallback"
 
 
+# DRAM traffic of validate_pass1 as counted by ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a reduced
+# config 4 (2^24 elements per tensor), per algorithmic byte; see profiles/validate_pass1_config4_2p24.md.
+# It stands only for the kernel sources it was captured on: their hash is checked.
+NCU_TRAFFIC = {"dram_bytes_per_algorithmic_byte": None, "sources_sha1": None}
+
+
+def kernel_sources_sha1():
+    import hashlib
+    h = hashlib.sha1()
+    for name in ("validate.cu", "plan.h", "plan.cu"):
+        with open(os.path.join(ROOT, "paper_2510_03760_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def ncu_traffic(alg_bytes):
+    if NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] is None or NCU_TRAFFIC["sources_sha1"] != kernel_sources_sha1():
+        return None
+    return NCU_TRAFFIC["dram_bytes_per_algorithmic_byte"] * alg_bytes
+
+
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) while a region runs."""
@@ -334,15 +355,7 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     kern_avg_ms = sum(kern_ms) / len(kern_ms)
     achieved = alg_bytes / (kern_avg_ms * 1e-3) / 1e9
-    traffic = None   # set from an ncu capture of this kernel version, see profiles/
-    tpath = os.path.join(ROOT, "profiles", "validate_pass1_traffic.json")
-    if os.path.exists(tpath):
-        try:
-            tj = json.load(open(tpath))
-            if tj.get("workload") == args.workload:
-                traffic = tj.get("dram_bytes_per_launch")
-        except Exception:
-            traffic = None
+    traffic = ncu_traffic(alg_bytes) if args.workload == "config4" else None
     roofline = {"kernel": "validate_pass1", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": UNIT,
                 "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": traffic,
                 "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms_avg": kern_avg_ms,
