@@ -320,7 +320,7 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
             for (int e = 0; e < E::kPerVec; ++e) {
                 const int i = v * E::kPerVec + e;
                 const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
-                cnt += (d > tol[i]) ? 1u : 0u;
+                cnt += __float_as_uint(__fsub_rn(tol[i], d)) >> 31;       // sign of tol - d: set iff d > tol
                 ma = fmaxf(ma, d);
                 sse = fmaf(d, d, sse);
                 trig |= d > __fmul_rz(mlo, fabsf(r[i]));
