@@ -262,6 +262,10 @@ __device__ __forceinline__ void ring_release(Ring& g, int lane) {
     g.advance();
 }
 
+// IEEE division, kept out of line: the walks below name it at 16 unrolled positions and run it
+// at one or two of them, so its body would only bloat the hot loop's instruction footprint.
+__device__ __noinline__ float div_rn(float a, float b) { return __fdiv_rn(a, b); }
+
 constexpr float kInf = __builtin_huge_valf();
 constexpr float kShrink = 0.99999904632568359375f;      // 1 - 2^-20
 
@@ -366,7 +370,7 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
                     const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
                     const float ar = fabsf(r[i]);
                     if (ar != 0.f && d > __fmul_rz(lo, ar)) {
-                        const float q = __fdiv_rn(d, ar);
+                        const float q = div_rn(d, ar);
                         if (q > mt) { mt = q; lo = __fmul_rz(mt, kShrink); }
                     }
                 }
