@@ -347,3 +347,150 @@ int oracle_fitness(const float* times, uint64_t n_cand, uint32_t trials,
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Other run-time statistics.  Section 4.3 says the run times over the repeated
+// runs are averaged, Appendix A.7.1 that their median is taken; both are
+// offered, with the minimum and a trimmed mean, and with the option to leave
+// out the first `warmup` runs.  Definitions (binary32 in, binary32 out):
+//   mean          sum of the kept runs, accumulated in binary64 in run order,
+//                 divided by their count in binary64, rounded once to binary32
+//   min           the smallest kept run
+//   trimmed mean  the kept runs sorted ascending, `trim` dropped at each end,
+//                 the rest summed in binary64 in ascending order, divided by
+//                 their count, rounded once to binary32
+// Speedup = baseline statistic / candidate statistic (one binary32 division),
+// the baseline's statistic being of the same kind.
+// ---------------------------------------------------------------------------
+enum { STAT_MEDIAN = 0, STAT_MEAN = 1, STAT_MIN = 2, STAT_TRIMMED_MEAN = 3 };
+
+static bool row_statistic(const float* row, uint32_t trials, int stat, uint32_t warmup, uint32_t trim, float* value) {
+    if (warmup >= trials) return false;
+    std::vector<float> v(row + warmup, row + trials);
+    for (float x : v) if (!(std::isfinite(x) && x > 0.0f)) return false;
+    const size_t m = v.size();
+    switch (stat) {
+        case STAT_MEDIAN: return row_median(v.data(), static_cast<uint32_t>(m), value);
+        case STAT_MEAN: {
+            double sum = 0.0;
+            for (float x : v) sum += static_cast<double>(x);
+            *value = static_cast<float>(sum / static_cast<double>(m));
+            return true;
+        }
+        case STAT_MIN: {
+            float lo = v[0];
+            for (float x : v) if (x < lo) lo = x;
+            *value = lo;
+            return true;
+        }
+        case STAT_TRIMMED_MEAN: {
+            if (2ull * trim >= m) return false;
+            std::sort(v.begin(), v.end());
+            double sum = 0.0;
+            for (size_t i = trim; i < m - trim; ++i) sum += static_cast<double>(v[i]);
+            *value = static_cast<float>(sum / static_cast<double>(m - 2ull * trim));
+            return true;
+        }
+        default: return false;
+    }
+}
+
+extern "C" int oracle_fitness_ex(const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
+                                 uint32_t base_trials, const uint32_t* pass, int stat, uint32_t warmup, uint32_t trim,
+                                 oracle_fit* out) {
+    if (trials == 0 || base_trials == 0 || stat < 0 || stat > 3) return -1;
+    if (warmup >= trials || warmup >= base_trials) return -1;
+    if (stat == STAT_TRIMMED_MEAN && (2ull * trim >= trials - warmup || 2ull * trim >= base_trials - warmup)) return -1;
+    float base_value = 0.0f;
+    const bool base_ok = row_statistic(base_times, base_trials, stat, warmup, trim, &base_value);
+    for (uint64_t i = 0; i < n_cand; ++i) {
+        oracle_fit f{};
+        float val = 0.0f;
+        const bool ok = row_statistic(times + i * static_cast<uint64_t>(trials), trials, stat, warmup, trim, &val);
+        if (!ok) { f.status = 1u; }
+        else if (!base_ok) { f.status = 2u; f.median_ms = val; }
+        else {
+            f.median_ms = val;
+            const bool passed = (pass == nullptr) || (pass[i] != 0u);
+            if (passed) { f.valid = 1u; f.speedup = base_value / val; }
+        }
+        out[i] = f;
+    }
+    return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Population summary: the paper's reporting metrics (Section 5.1 "Evaluation
+// Metric"; the speedup-range table of Appendix A.5) from the per-candidate
+// fitness records of one or several independent runs.
+//   best[r][k]   largest speedup among the valid candidates of kernel k in run
+//                r (0 if none is valid)
+//   per run      median over the kernels of max(best, 1.0): a kernel without a
+//                candidate that beats the baseline counts as 1.0
+//   median_speedup  mean of the per-run medians (binary64 sum in run order,
+//                one rounding to binary32): "averaged over three runs"
+//   validity     valid candidates / candidates (Pass@1), binary32 division of
+//                the two counts converted to binary64 and rounded once
+//   speedup_count   kernels whose best over all runs exceeds 1.0
+//   hist[5]      kernels by their best over all runs: < 1, [1, 2), [2, 5),
+//                [5, 10), >= 10 (the table prints "<1.0, 1.0~2.0, 2.0~5.0,
+//                5.0~10.0, >10.0"; which side the boundaries fall is this
+//                library's reading)
+// ---------------------------------------------------------------------------
+struct oracle_summary_rec {
+    float median_speedup;
+    float validity;
+    uint32_t n_valid;
+    uint32_t n_cand;
+    uint32_t speedup_count;
+    uint32_t hist[5];
+    uint32_t n_kernel;
+    uint32_t n_run;
+};
+
+extern "C" int oracle_summary(const oracle_fit* fits, const uint32_t* kernel_of, const uint32_t* run_of, uint64_t n_cand,
+                              uint32_t n_kernel, uint32_t n_run, oracle_summary_rec* out, float* best /* n_run*n_kernel */,
+                              float* run_median /* n_run */) {
+    if (n_kernel == 0 || n_run == 0) return -1;
+    std::vector<float> b(static_cast<size_t>(n_run) * n_kernel, 0.0f);
+    uint32_t n_valid = 0;
+    for (uint64_t i = 0; i < n_cand; ++i) {
+        const uint32_t k = kernel_of[i], r = run_of ? run_of[i] : 0u;
+        if (k >= n_kernel || r >= n_run) return -1;
+        if (!fits[i].valid) continue;
+        ++n_valid;
+        float& slot = b[static_cast<size_t>(r) * n_kernel + k];
+        if (fits[i].speedup > slot) slot = fits[i].speedup;
+    }
+    double sum = 0.0;
+    for (uint32_t r = 0; r < n_run; ++r) {
+        std::vector<float> v(n_kernel);
+        for (uint32_t k = 0; k < n_kernel; ++k) {
+            const float x = b[static_cast<size_t>(r) * n_kernel + k];
+            v[k] = x > 1.0f ? x : 1.0f;
+        }
+        std::sort(v.begin(), v.end());
+        float med;
+        if (n_kernel & 1u) med = v[n_kernel / 2];
+        else { const float s = v[n_kernel / 2 - 1] + v[n_kernel / 2]; med = 0.5f * s; }
+        if (run_median) run_median[r] = med;
+        sum += static_cast<double>(med);
+    }
+    oracle_summary_rec s{};
+    s.median_speedup = static_cast<float>(sum / static_cast<double>(n_run));
+    s.n_valid = n_valid;
+    s.n_cand = static_cast<uint32_t>(n_cand);
+    s.validity = n_cand ? static_cast<float>(static_cast<double>(n_valid) / static_cast<double>(n_cand)) : 0.0f;
+    s.n_kernel = n_kernel;
+    s.n_run = n_run;
+    for (uint32_t k = 0; k < n_kernel; ++k) {
+        float top = 0.0f;
+        for (uint32_t r = 0; r < n_run; ++r) top = std::max(top, b[static_cast<size_t>(r) * n_kernel + k]);
+        if (top > 1.0f) ++s.speedup_count;
+        const int bin = top < 1.0f ? 0 : top < 2.0f ? 1 : top < 5.0f ? 2 : top < 10.0f ? 3 : 4;
+        ++s.hist[bin];
+    }
+    if (best) std::memcpy(best, b.data(), b.size() * sizeof(float));
+    *out = s;
+    return 0;
+}

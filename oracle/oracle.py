@@ -17,7 +17,11 @@ RESULT_DTYPE = np.dtype(
      ("max_rel", "<f4"), ("flags", "<u4"), ("pass", "<u4")], align=True)
 FIT_DTYPE = np.dtype(
     [("median_ms", "<f4"), ("speedup", "<f4"), ("valid", "<u4"), ("status", "<u4")], align=True)
-assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16
+SUMMARY_DTYPE = np.dtype(
+    [("median_speedup", "<f4"), ("validity", "<f4"), ("n_valid", "<u4"), ("n_cand", "<u4"), ("speedup_count", "<u4"),
+     ("hist", "<u4", (5,)), ("n_kernel", "<u4"), ("n_run", "<u4")], align=True)
+assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16 and SUMMARY_DTYPE.itemsize == 48
+STAT_MEDIAN, STAT_MEAN, STAT_MIN, STAT_TRIMMED_MEAN = 0, 1, 2, 3
 
 _lib = None
 
@@ -48,6 +52,12 @@ def lib():
         L.oracle_group_pass.restype = None
         L.oracle_fitness.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
         L.oracle_fitness.restype = C.c_int
+        L.oracle_fitness_ex.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_uint32, C.c_void_p, C.c_int,
+                                        C.c_uint32, C.c_uint32, C.c_void_p]
+        L.oracle_fitness_ex.restype = C.c_int
+        L.oracle_summary.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
+                                     C.c_void_p, C.c_void_p]
+        L.oracle_summary.restype = C.c_int
         _lib = L
     return _lib
 
@@ -160,3 +170,38 @@ def fitness(times, base_times, passed=None):
     if rc != 0:
         raise ValueError("oracle_fitness: status %d" % rc)
     return out
+
+
+def fitness_ex(times, base_times, passed=None, stat=STAT_MEDIAN, warmup=0, trim=0):
+    """fitness() with the run-time statistic chosen (median, mean, min, trimmed mean), the first
+    `warmup` runs left out and, for the trimmed mean, `trim` runs dropped at each end."""
+    times = np.ascontiguousarray(times, dtype=np.float32)
+    base = np.ascontiguousarray(base_times, dtype=np.float32)
+    assert times.ndim == 2 and base.ndim == 1
+    n_cand, trials = times.shape
+    p = None
+    if passed is not None:
+        p = np.ascontiguousarray(passed, dtype=np.uint32)
+        assert p.shape == (n_cand,)
+    out = np.zeros(n_cand, dtype=FIT_DTYPE)
+    rc = lib().oracle_fitness_ex(_ptr(times), n_cand, trials, _ptr(base), base.size, _ptr(p) if p is not None else None,
+                                 int(stat), int(warmup), int(trim), _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_fitness_ex: status %d" % rc)
+    return out
+
+
+def summary(fits, kernel_of, n_kernel, run_of=None, n_run=1):
+    """Reporting metrics of a population.  Returns (SUMMARY_DTYPE scalar, best [n_run, n_kernel],
+    run_median [n_run])."""
+    fits = np.ascontiguousarray(fits, dtype=FIT_DTYPE)
+    k = np.ascontiguousarray(kernel_of, dtype=np.uint32)
+    r = np.ascontiguousarray(run_of, dtype=np.uint32) if run_of is not None else None
+    out = np.zeros(1, dtype=SUMMARY_DTYPE)
+    best = np.zeros((int(n_run), int(n_kernel)), dtype=np.float32)
+    med = np.zeros(int(n_run), dtype=np.float32)
+    rc = lib().oracle_summary(_ptr(fits), _ptr(k), _ptr(r) if r is not None else None, fits.size, int(n_kernel), int(n_run),
+                              _ptr(out), _ptr(best), _ptr(med))
+    if rc != 0:
+        raise ValueError("oracle_summary: status %d" % rc)
+    return out[0], best, med
