@@ -194,10 +194,62 @@ EVO_API int evo_fitness(evo_ctx* ctx, const float* times /* device */, uint64_t 
                 const float* base_times /* device */, uint32_t base_trials,
                 const uint32_t* pass /* device, optional */, evo_fit* out /* device */, void* stream);
 
+/*
+ * evo_fitness_ex - evo_fitness with the run-time statistic chosen.
+ * Paper: Section 4.3 says the run times are averaged, Appendix A.7.1 that their median is
+ * taken; this call offers both, the minimum and a trimmed mean, and can leave out the first
+ * `warmup` runs of every row (and of the baseline).  The statistic is reported in
+ * evo_fit.median_ms; speedup = baseline statistic / candidate statistic, of the same kind.
+ *   EVO_STAT_MEDIAN        as evo_fitness
+ *   EVO_STAT_MEAN          binary64 sum of the kept runs in run order / their count, rounded once to binary32
+ *   EVO_STAT_MIN           the smallest kept run
+ *   EVO_STAT_TRIMMED_MEAN  kept runs in ascending order, `trim` dropped at each end, binary64 sum of the rest in
+ *                          that order / their count, rounded once to binary32
+ * warmup < trials and < base_trials; 2 * trim < kept runs (trimmed mean only; ignored otherwise).
+ * Errors: as evo_fitness.
+ */
+enum { EVO_STAT_MEDIAN = 0, EVO_STAT_MEAN = 1, EVO_STAT_MIN = 2, EVO_STAT_TRIMMED_MEAN = 3 };
+EVO_API int evo_fitness_ex(evo_ctx* ctx, const float* times /* device */, uint64_t n_cand, uint32_t trials,
+                           const float* base_times /* device */, uint32_t base_trials, const uint32_t* pass /* device, optional */,
+                           int stat, uint32_t warmup, uint32_t trim, evo_fit* out /* device */, void* stream);
+
 /* evo_fitness for host arrays (all four pointers are HOST addresses); synchronises the stream. */
 EVO_API int evo_fitness_host(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials,
                      const float* base_times, uint32_t base_trials,
                      const uint32_t* pass, evo_fit* out, void* stream);
+
+/*
+ * evo_summary - the reporting metrics of a population from its evo_fit records.
+ * Paper: Section 5.1 "Evaluation Metric" (the median speedup across kernels, 1.0 for a kernel
+ * where no candidate beats the baseline, averaged over the independent runs; Pass@1 = the
+ * share of trials that yield a valid kernel); Appendix A.5 (kernels counted by speedup range).
+ *   best[r][k]      largest speedup among the valid candidates of kernel k in run r (0 if none)
+ *   run_median[r]   median over the kernels of max(best[r][k], 1.0) (middle value, or
+ *                   0.5 * (a + b) of the two middle ones, binary32)
+ *   median_speedup  mean of the run medians (binary64 sum in run order, rounded once)
+ *   validity        n_valid / n_cand (binary64 quotient of the counts, rounded once)
+ *   speedup_count   kernels whose best over all runs exceeds 1.0
+ *   hist[0..4]      kernels by their best over all runs: < 1, [1, 2), [2, 5), [5, 10), >= 10
+ *                   (the paper prints the ranges without saying where the boundaries belong)
+ * fits       : device, n_cand records (as written by evo_fitness).
+ * kernel_of  : device, n_cand kernel ids in [0, n_kernel).
+ * run_of     : device, n_cand run ids in [0, n_run); NULL = all in run 0.
+ * out        : device, one record.
+ * best       : device, n_run * n_kernel floats, written (it doubles as the call's workspace).
+ * run_median : device, n_run floats, optional.
+ * 1 <= n_kernel <= 8192, 1 <= n_run <= 1024.  An id out of range makes the next evo_check
+ * return EVO_ERR_ARG (the record is skipped).  Errors: EVO_ERR_ARG, EVO_ERR_ALIGN, EVO_ERR_CUDA.
+ */
+typedef struct {
+    float median_speedup, validity;
+    uint32_t n_valid, n_cand, speedup_count;
+    uint32_t hist[5];
+    uint32_t n_kernel, n_run;
+} evo_summary_rec;         /* 48 bytes */
+EVO_API int evo_summary(evo_ctx* ctx, const evo_fit* fits /* device */, const uint32_t* kernel_of /* device */,
+                        const uint32_t* run_of /* device, optional */, uint64_t n_cand, uint32_t n_kernel, uint32_t n_run,
+                        evo_summary_rec* out /* device */, float* best /* device */, float* run_median /* device, optional */,
+                        void* stream);
 
 /*
  * evo_validate_static - evo_validate for callers that cannot allocate device memory.
@@ -273,7 +325,8 @@ EVO_API int evo_set_timing_events(evo_ctx* ctx, void* start, void* stop);
  * into shared memory that does not land within 2 s makes the CTA stop, raise a status word
  * and return); when that happened, evo_validate's results carry EVO_FLAG_INCOMPLETE with
  * pass = 0, and this call returns EVO_ERR_TIMEOUT once and clears the word.  The *_host
- * variants do this check themselves.  (The paper has no counterpart.)
+ * variants do this check themselves.  It also reports, as EVO_ERR_ARG, an id out of range
+ * that evo_summary met on the device.  (The paper has no counterpart.)
  * Errors: EVO_ERR_ARG, EVO_ERR_CUDA, EVO_ERR_TIMEOUT.
  */
 EVO_API int evo_check(evo_ctx* ctx, void* stream);

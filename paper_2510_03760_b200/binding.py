@@ -16,7 +16,12 @@ RESULT_DTYPE = np.dtype(
 FIT_DTYPE = np.dtype(
     [("median_ms", "<f4"), ("speedup", "<f4"), ("valid", "<u4"), ("status", "<u4")], align=True)
 _DESC_DTYPE = np.dtype([("n", "<u8"), ("ref", "<u8"), ("dtype", "<i4"), ("group", "<u4")], align=True)
+SUMMARY_DTYPE = np.dtype(
+    [("median_speedup", "<f4"), ("validity", "<f4"), ("n_valid", "<u4"), ("n_cand", "<u4"), ("speedup_count", "<u4"),
+     ("hist", "<u4", (5,)), ("n_kernel", "<u4"), ("n_run", "<u4")], align=True)
+EVO_STAT_MEDIAN, EVO_STAT_MEAN, EVO_STAT_MIN, EVO_STAT_TRIMMED_MEAN = 0, 1, 2, 3
 assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16 and _DESC_DTYPE.itemsize == 24
+assert SUMMARY_DTYPE.itemsize == 48
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libevo.so")
 _lib = None
@@ -67,6 +72,10 @@ def load_library():
         fn = getattr(L, name)
         fn.argtypes = [vp, vp, u64, u32, vp, u32, vp, vp, vp]
         fn.restype = i32
+    L.evo_fitness_ex.argtypes = [vp, vp, u64, u32, vp, u32, vp, i32, u32, u32, vp, vp]
+    L.evo_fitness_ex.restype = i32
+    L.evo_summary.argtypes = [vp, vp, vp, vp, u64, u32, u32, vp, vp, vp, vp]
+    L.evo_summary.restype = i32
     _lib = L
     return L
 
@@ -241,9 +250,10 @@ def evo_validate_host(cands, refs, atol, rtol, groups=None, n_group=0, device=No
     return results, gp
 
 
-def evo_fitness(times, base_times, passed=None, out=None, stream=None, ctx=None):
+def evo_fitness(times, base_times, passed=None, out=None, stream=None, ctx=None, stat=EVO_STAT_MEDIAN, warmup=0, trim=0):
     """times [n_cand, trials] float32 CUDA, base_times [base_trials] float32 CUDA, passed
-    optional int32/uint32 [n_cand].  Returns a uint8 CUDA tensor of n_cand x 16 bytes (evo_fit)."""
+    optional int32/uint32 [n_cand].  Returns a uint8 CUDA tensor of n_cand x 16 bytes (evo_fit).
+    `stat`, `warmup`, `trim` choose the run-time statistic (evo_fitness_ex)."""
     if times.dtype != torch.float32 or base_times.dtype != torch.float32 or times.dim() != 2:
         raise ValueError("times must be a 2-D float32 tensor and base_times float32")
     if not (times.is_contiguous() and base_times.is_contiguous()):
@@ -252,10 +262,40 @@ def evo_fitness(times, base_times, passed=None, out=None, stream=None, ctx=None)
     ctx = ctx or default_context(times.device.index)
     if out is None:
         out = torch.empty((n_cand, FIT_DTYPE.itemsize), dtype=torch.uint8, device=times.device)
-    st = load_library().evo_fitness(ctx._h, _dev_ptr(times), n_cand, trials, _dev_ptr(base_times), base_times.numel(),
-                                    _dev_ptr(passed), _dev_ptr(out), _stream_ptr(stream, times.device))
+    L = load_library()
+    if stat == EVO_STAT_MEDIAN and warmup == 0:
+        st = L.evo_fitness(ctx._h, _dev_ptr(times), n_cand, trials, _dev_ptr(base_times), base_times.numel(),
+                           _dev_ptr(passed), _dev_ptr(out), _stream_ptr(stream, times.device))
+    else:
+        st = L.evo_fitness_ex(ctx._h, _dev_ptr(times), n_cand, trials, _dev_ptr(base_times), base_times.numel(),
+                              _dev_ptr(passed), int(stat), int(warmup), int(trim), _dev_ptr(out),
+                              _stream_ptr(stream, times.device))
     ctx.check(st)
     return out
+
+
+def evo_summary(fits, kernel_of, n_kernel, run_of=None, n_run=1, stream=None, ctx=None):
+    """Reporting metrics of a population: `fits` is the uint8 CUDA tensor evo_fitness returned,
+    `kernel_of` (and optionally `run_of`) int32 CUDA tensors with one id per candidate.  Returns
+    (summary: uint8 CUDA tensor of 48 bytes, see summary_to_numpy; best: float32 [n_run, n_kernel];
+    run_median: float32 [n_run])."""
+    n_cand = fits.shape[0]
+    dev = fits.device
+    ctx = ctx or default_context(dev.index)
+    for t in (kernel_of, run_of):
+        if t is not None and (t.dtype not in (torch.int32, torch.uint32) or t.numel() != n_cand or not t.is_contiguous()):
+            raise ValueError("kernel_of / run_of must be contiguous 32-bit integer tensors with one entry per candidate")
+    out = torch.empty(SUMMARY_DTYPE.itemsize, dtype=torch.uint8, device=dev)
+    best = torch.empty((int(n_run), int(n_kernel)), dtype=torch.float32, device=dev)
+    med = torch.empty(int(n_run), dtype=torch.float32, device=dev)
+    st = load_library().evo_summary(ctx._h, _dev_ptr(fits), _dev_ptr(kernel_of), _dev_ptr(run_of), n_cand, int(n_kernel),
+                                    int(n_run), _dev_ptr(out), _dev_ptr(best), _dev_ptr(med), _stream_ptr(stream, dev))
+    ctx.check(st)
+    return out, best, med
+
+
+def summary_to_numpy(summary):
+    return summary.cpu().numpy().view(SUMMARY_DTYPE)[0]
 
 
 def evo_fitness_host(times, base_times, passed=None, device=None, stream=None, ctx=None):

@@ -85,7 +85,9 @@ int sync_and_check(evo_ctx* ctx, cudaStream_t stream, const char* who) {
     EVO_CUDA_TRY(ctx, cudaMemcpy(&word, status_word(ctx), sizeof word, cudaMemcpyDeviceToHost));
     if (word == 0) return EVO_OK;
     EVO_CUDA_TRY(ctx, cudaMemset(status_word(ctx), 0, sizeof word));
-    return fail(ctx, EVO_ERR_TIMEOUT, "%s: a device-side wait ran out (status word 0x%x); results are marked incomplete", who, word);
+    if (word & 3u)
+        return fail(ctx, EVO_ERR_TIMEOUT, "%s: a device-side wait ran out (status word 0x%x); results are marked incomplete", who, word);
+    return fail(ctx, EVO_ERR_ARG, "%s: a kernel or run id was out of range (status word 0x%x); that record was skipped", who, word);
 }
 
 }  // namespace evo

@@ -18,28 +18,69 @@ constexpr uint32_t kMaxTrials = 4096;
 
 struct RowMedian { float median; uint32_t ok; };
 
-// Median of row[0..trials) held in shared memory, computed by one warp.  ok = 0 when a
-// time is NaN, Inf or not positive.  All lanes return the same value.
-__device__ RowMedian warp_median(const float* row, uint32_t trials, int lane, float* slot /* 2 floats, warp-private */) {
+// Statistic of row[0..m) held in shared memory, computed by one warp.  ok = 0 when a time is
+// NaN, Inf or not positive.  All lanes return the same value.
+//   median        middle order statistic, or 0.5 * (a + b) of the two middle ones (binary32)
+//   mean          binary64 sum in run order, one division, one rounding to binary32
+//   min           the smallest run
+//   trimmed mean  runs ranked, `trim` dropped at each end, binary64 sum in ascending order
+// Order statistics come from rank counting (rank of x_i = number of j with x_j < x_i, or
+// x_j == x_i and j < i): no sort, and the result does not depend on the order of the runs.
+// The sums are taken by one lane in a fixed order, so they are reproducible bit for bit.
+__device__ RowMedian warp_statistic(const float* row, uint32_t m, int stat, uint32_t trim, int lane,
+                                    float* slot /* 2 floats */, float* sorted /* m floats, trimmed mean only */) {
     const unsigned full = 0xffffffffu;
     bool bad = false;
-    for (uint32_t i = lane; i < trials; i += 32) {
+    for (uint32_t i = lane; i < m; i += 32) {
         const float x = row[i];
         bad |= !(x > 0.f && x < __int_as_float(0x7f800000));
     }
     if (__any_sync(full, bad)) return RowMedian{0.f, 0u};
-    const uint32_t lo = (trials - 1) / 2, hi = trials / 2;     // equal when trials is odd
-    for (uint32_t i = lane; i < trials; i += 32) {
+    if (stat == EVO_STAT_MEAN) {
+        if (lane == 0) {
+            double sum = 0.0;
+            for (uint32_t i = 0; i < m; ++i) sum += static_cast<double>(row[i]);
+            slot[0] = static_cast<float>(sum / static_cast<double>(m));
+        }
+        __syncwarp();
+        const float v = slot[0];
+        __syncwarp();
+        return RowMedian{v, 1u};
+    }
+    if (stat == EVO_STAT_MIN) {
+        float lo = __int_as_float(0x7f800000);
+        for (uint32_t i = lane; i < m; i += 32) lo = fminf(lo, row[i]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) lo = fminf(lo, __shfl_xor_sync(full, lo, o));
+        return RowMedian{lo, 1u};
+    }
+    const uint32_t lo = (m - 1) / 2, hi = m / 2;     // equal when m is odd
+    for (uint32_t i = lane; i < m; i += 32) {
         const float x = row[i];
         uint32_t rank = 0;
-        for (uint32_t j = 0; j < trials; ++j) {
+        for (uint32_t j = 0; j < m; ++j) {
             const float y = row[j];
             rank += (y < x || (y == x && j < i)) ? 1u : 0u;
         }
-        if (rank == lo) slot[0] = x;
-        if (rank == hi) slot[1] = x;
+        if (stat == EVO_STAT_TRIMMED_MEAN) {
+            sorted[rank] = x;
+        } else {
+            if (rank == lo) slot[0] = x;
+            if (rank == hi) slot[1] = x;
+        }
     }
     __syncwarp();
+    if (stat == EVO_STAT_TRIMMED_MEAN) {
+        if (lane == 0) {
+            double sum = 0.0;
+            for (uint32_t i = trim; i < m - trim; ++i) sum += static_cast<double>(sorted[i]);
+            slot[0] = static_cast<float>(sum / static_cast<double>(m - 2 * trim));
+        }
+        __syncwarp();
+        const float v = slot[0];
+        __syncwarp();
+        return RowMedian{v, 1u};
+    }
     const float a = slot[0], b = slot[1];
     __syncwarp();
     const float med = (lo == hi) ? a : __fmul_rn(0.5f, __fadd_rn(a, b));
@@ -47,19 +88,22 @@ __device__ RowMedian warp_median(const float* row, uint32_t trials, int lane, fl
 }
 
 __global__ void __launch_bounds__(kWarpsPerCta * 32)
-fitness_kernel(const float* __restrict__ times, uint64_t n_rows, uint32_t trials,
-               const RowMedian* __restrict__ base /* nullptr: write the row's median to base_out */,
+fitness_kernel(const float* __restrict__ times, uint64_t n_rows, uint32_t trials, int stat, uint32_t warmup, uint32_t trim,
+               const RowMedian* __restrict__ base /* nullptr: write the row's statistic to base_out */,
                RowMedian* __restrict__ base_out, const uint32_t* __restrict__ pass, evo_fit* __restrict__ out) {
     extern __shared__ float smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float* row = smem + static_cast<size_t>(warp) * (trials + 2);
-    float* slot = row + trials;
+    const uint32_t m = trials - warmup;                                   // runs that count
+    const uint32_t per_warp = (stat == EVO_STAT_TRIMMED_MEAN ? 2 * m : m) + 2;
+    float* row = smem + static_cast<size_t>(warp) * per_warp;
+    float* slot = row + m;
+    float* sorted = slot + 2;
     const uint64_t r = static_cast<uint64_t>(blockIdx.x) * kWarpsPerCta + warp;
     if (r >= n_rows) return;
-    const float* src = times + r * trials;
-    for (uint32_t i = lane; i < trials; i += 32) row[i] = src[i];
+    const float* src = times + r * trials + warmup;
+    for (uint32_t i = lane; i < m; i += 32) row[i] = src[i];
     __syncwarp();
-    const RowMedian med = warp_median(row, trials, lane, slot);
+    const RowMedian med = warp_statistic(row, m, stat, trim, lane, slot, sorted);
     if (lane != 0) return;
     if (!base) { *base_out = med; return; }
     const RowMedian b = *base;
@@ -75,27 +119,39 @@ fitness_kernel(const float* __restrict__ times, uint64_t n_rows, uint32_t trials
     out[r] = f;
 }
 
+size_t smem_bytes(uint32_t trials, int stat, uint32_t warmup) {
+    const size_t m = trials - warmup;
+    return ((stat == EVO_STAT_TRIMMED_MEAN ? 2 * m : m) + 2) * sizeof(float) * kWarpsPerCta;
+}
+
 int fitness_device(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
-                   uint32_t base_trials, const uint32_t* pass, evo_fit* out, cudaStream_t stream) {
+                   uint32_t base_trials, const uint32_t* pass, int stat, uint32_t warmup, uint32_t trim, evo_fit* out,
+                   cudaStream_t stream) {
     RowMedian* d_base = static_cast<RowMedian*>(ctx->d_small);
-    const size_t smem_base = (static_cast<size_t>(base_trials) + 2) * sizeof(float) * kWarpsPerCta;
-    const size_t smem_rows = (static_cast<size_t>(trials) + 2) * sizeof(float) * kWarpsPerCta;
+    const size_t smem_base = smem_bytes(base_trials, stat, warmup), smem_rows = smem_bytes(trials, stat, warmup);
     if (std::max(smem_base, smem_rows) > 48 * 1024)
         EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(fitness_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>((kMaxTrials + 2) * sizeof(float) * kWarpsPerCta)));
-    fitness_kernel<<<1, kWarpsPerCta * 32, smem_base, stream>>>(base_times, 1, base_trials, nullptr, d_base, nullptr, nullptr);
+                                               static_cast<int>(smem_bytes(kMaxTrials, EVO_STAT_TRIMMED_MEAN, 0))));
+    fitness_kernel<<<1, kWarpsPerCta * 32, smem_base, stream>>>(base_times, 1, base_trials, stat, warmup, trim, nullptr, d_base,
+                                                               nullptr, nullptr);
     ctx->launches += 1;
     EVO_CUDA_TRY(ctx, cudaGetLastError());
     if (n_cand == 0) return EVO_OK;
     const unsigned grid = static_cast<unsigned>((n_cand + kWarpsPerCta - 1) / kWarpsPerCta);
-    fitness_kernel<<<grid, kWarpsPerCta * 32, smem_rows, stream>>>(times, n_cand, trials, d_base, nullptr, pass, out);
+    fitness_kernel<<<grid, kWarpsPerCta * 32, smem_rows, stream>>>(times, n_cand, trials, stat, warmup, trim, d_base, nullptr,
+                                                                  pass, out);
     ctx->launches += 1;
     EVO_CUDA_TRY(ctx, cudaGetLastError());
     return EVO_OK;
 }
 
 int check_args(evo_ctx* ctx, const char* who, const float* times, uint64_t n_cand, uint32_t trials,
-               const float* base_times, uint32_t base_trials, evo_fit* out) {
+               const float* base_times, uint32_t base_trials, int stat, uint32_t warmup, uint32_t trim, evo_fit* out) {
+    if (stat < EVO_STAT_MEDIAN || stat > EVO_STAT_TRIMMED_MEAN) return evo::fail(ctx, EVO_ERR_ARG, "%s: stat %d", who, stat);
+    if (warmup >= trials || warmup >= base_trials)
+        return evo::fail(ctx, EVO_ERR_ARG, "%s: warmup must leave at least one run", who);
+    if (stat == EVO_STAT_TRIMMED_MEAN && (2ull * trim >= trials - warmup || 2ull * trim >= base_trials - warmup))
+        return evo::fail(ctx, EVO_ERR_ARG, "%s: trim must leave at least one run", who);
     if (trials == 0 || base_trials == 0 || trials > kMaxTrials || base_trials > kMaxTrials)
         return evo::fail(ctx, EVO_ERR_ARG, "%s: trials and base_trials must be in [1, %u]", who, kMaxTrials);
     if (!base_times || (n_cand > 0 && (!times || !out)))
@@ -108,20 +164,27 @@ int check_args(evo_ctx* ctx, const char* who, const float* times, uint64_t n_can
 
 }  // namespace
 
-extern "C" int evo_fitness(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
-                           uint32_t base_trials, const uint32_t* pass, evo_fit* out, void* stream) {
+extern "C" int evo_fitness_ex(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
+                              uint32_t base_trials, const uint32_t* pass, int stat, uint32_t warmup, uint32_t trim,
+                              evo_fit* out, void* stream) {
     if (!ctx) return EVO_ERR_ARG;
-    int st = check_args(ctx, "evo_fitness", times, n_cand, trials, base_times, base_trials, out);
+    int st = check_args(ctx, "evo_fitness", times, n_cand, trials, base_times, base_trials, stat, warmup, trim, out);
     if (st != EVO_OK) return st;
     evo::DeviceGuard guard(ctx->device);
     if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
-    return fitness_device(ctx, times, n_cand, trials, base_times, base_trials, pass, out, static_cast<cudaStream_t>(stream));
+    return fitness_device(ctx, times, n_cand, trials, base_times, base_trials, pass, stat, warmup, trim, out,
+                          static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int evo_fitness(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
+                           uint32_t base_trials, const uint32_t* pass, evo_fit* out, void* stream) {
+    return evo_fitness_ex(ctx, times, n_cand, trials, base_times, base_trials, pass, EVO_STAT_MEDIAN, 0, 0, out, stream);
 }
 
 extern "C" int evo_fitness_host(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
                                 uint32_t base_trials, const uint32_t* pass, evo_fit* out, void* stream_) {
     if (!ctx) return EVO_ERR_ARG;
-    int st = check_args(ctx, "evo_fitness_host", times, n_cand, trials, base_times, base_trials, out);
+    int st = check_args(ctx, "evo_fitness_host", times, n_cand, trials, base_times, base_trials, EVO_STAT_MEDIAN, 0, 0, out);
     if (st != EVO_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     evo::DeviceGuard guard(ctx->device);
@@ -137,7 +200,7 @@ extern "C" int evo_fitness_host(evo_ctx* ctx, const float* times, uint64_t n_can
     EVO_CUDA_TRY(ctx, cudaMemcpyAsync(base + o_base, base_times, b_base, cudaMemcpyHostToDevice, stream));
     if (pass && n_cand) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(base + o_pass, pass, n_cand * 4, cudaMemcpyHostToDevice, stream));
     st = fitness_device(ctx, reinterpret_cast<const float*>(base), n_cand, trials, reinterpret_cast<const float*>(base + o_base),
-                        base_trials, pass ? reinterpret_cast<const uint32_t*>(base + o_pass) : nullptr,
+                        base_trials, pass ? reinterpret_cast<const uint32_t*>(base + o_pass) : nullptr, EVO_STAT_MEDIAN, 0, 0,
                         reinterpret_cast<evo_fit*>(base + o_out), stream);
     if (st != EVO_OK) return st;
     if (n_cand) EVO_CUDA_TRY(ctx, cudaMemcpyAsync(out, base + o_out, n_cand * sizeof(evo_fit), cudaMemcpyDeviceToHost, stream));

@@ -57,3 +57,35 @@ def test_argument_errors(evo):
     assert L.evo_fitness(ctx._h, t.data_ptr(), 2, 4, t.data_ptr(), 5000, None, o.data_ptr(), None) == -1
     assert L.evo_fitness(ctx._h, None, 2, 4, t.data_ptr(), 4, None, o.data_ptr(), None) == -1
     assert L.evo_fitness(ctx._h, t.data_ptr(), 0, 4, t.data_ptr(), 4, None, None, None) == 0
+
+
+@pytest.mark.parametrize("stat", [0, 1, 2, 3])
+@pytest.mark.parametrize("trials", [1, 2, 7, 100, 129, 1000, 4096])
+def test_other_statistics_and_warmup(evo, stat, trials):
+    rng = np.random.default_rng(100 * stat + trials)
+    n = 19 if trials < 1000 else 4
+    times = (10.0 ** rng.uniform(-2, 2, (n, trials))).astype(np.float32)
+    times[1] = times[1, 0]
+    times[2, : trials // 2] = times[2, 0]
+    base_trials = max(1, trials // 2) if trials > 7 else trials
+    base = (1 + rng.random(base_trials)).astype(np.float32)
+    passed = rng.integers(0, 2, n)
+    for warmup in sorted({0, min(3, base_trials - 1)}):
+        kept = min(trials, base_trials) - warmup
+        for trim in sorted({0, (kept - 1) // 2, kept // 10}) if stat == 3 else [0]:
+            t = torch.from_numpy(times).cuda()
+            b = torch.from_numpy(base).cuda()
+            p = torch.from_numpy(passed.astype(np.int32)).cuda()
+            got = evo.fits_to_numpy(evo.evo_fitness(t, b, p, stat=stat, warmup=warmup, trim=trim))
+            want = oracle.fitness_ex(times, base, passed, stat=stat, warmup=warmup, trim=trim)
+            assert got.tobytes() == want.tobytes(), (stat, trials, warmup, trim)
+
+
+def test_statistics_with_bad_runs_and_bad_arguments(evo):
+    t = np.array([[1, 2, 3, 4], [1, np.nan, 3, 4], [np.nan, 2, 3, 4]], np.float32)
+    base = np.array([2, 2, 2, 2], np.float32)
+    got = evo.fits_to_numpy(evo.evo_fitness(torch.from_numpy(t).cuda(), torch.from_numpy(base).cuda(), stat=1, warmup=1))
+    assert got.tobytes() == oracle.fitness_ex(t, base, stat=1, warmup=1).tobytes()
+    for kw in (dict(stat=7), dict(stat=1, warmup=4), dict(stat=3, trim=2), dict(stat=3, warmup=2, trim=1)):
+        with pytest.raises(evo.EvoError):
+            evo.evo_fitness(torch.from_numpy(t).cuda(), torch.from_numpy(base).cuda(), **kw)
