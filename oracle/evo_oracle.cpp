@@ -494,3 +494,20 @@ extern "C" int oracle_summary(const oracle_fit* fits, const uint32_t* kernel_of,
     *out = s;
     return 0;
 }
+
+// ---------------------------------------------------------------------------
+// Elite selection (Section 4.2 "Population Management": the single-solution
+// strategy keeps the current best solution, elite preservation keeps a small
+// set of high-performing ones).  The k valid candidates with the largest
+// speedup, best first; equal speedups in order of their index.  Writes
+// min(k, number of valid candidates) indices, fills the rest with 0xffffffff.
+// ---------------------------------------------------------------------------
+extern "C" int oracle_select_elite(const oracle_fit* fits, uint64_t n_cand, uint32_t k, uint32_t* idx, uint32_t* count) {
+    std::vector<uint32_t> order;
+    for (uint64_t i = 0; i < n_cand; ++i) if (fits[i].valid) order.push_back(static_cast<uint32_t>(i));
+    std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return fits[a].speedup > fits[b].speedup; });
+    const uint32_t m = static_cast<uint32_t>(std::min<size_t>(k, order.size()));
+    for (uint32_t i = 0; i < k; ++i) idx[i] = i < m ? order[i] : 0xffffffffu;
+    *count = m;
+    return 0;
+}

@@ -58,6 +58,8 @@ def lib():
         L.oracle_summary.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
                                      C.c_void_p, C.c_void_p]
         L.oracle_summary.restype = C.c_int
+        L.oracle_select_elite.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p]
+        L.oracle_select_elite.restype = C.c_int
         _lib = L
     return _lib
 
@@ -205,3 +207,13 @@ def summary(fits, kernel_of, n_kernel, run_of=None, n_run=1):
     if rc != 0:
         raise ValueError("oracle_summary: status %d" % rc)
     return out[0], best, med
+
+
+def select_elite(fits, k):
+    """Indices of the k valid candidates with the largest speedup, best first (ties by index);
+    returns (idx [k] uint32, padded with 0xffffffff, and the number of real entries)."""
+    fits = np.ascontiguousarray(fits, dtype=FIT_DTYPE)
+    idx = np.zeros(int(k), dtype=np.uint32)
+    count = np.zeros(1, dtype=np.uint32)
+    lib().oracle_select_elite(_ptr(fits), fits.size, int(k), _ptr(idx), _ptr(count))
+    return idx, int(count[0])

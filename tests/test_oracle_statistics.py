@@ -147,3 +147,29 @@ def test_summary_floor_boundaries_and_errors():
         oracle.summary(_fits([1], [1.0]), [3], 3)
     with pytest.raises(ValueError):
         oracle.summary(_fits([1], [1.0]), [0], 3, run_of=[1], n_run=1)
+
+
+def test_elite_selection_against_lexsort_argmax_and_brute_force():
+    rng = np.random.default_rng(33)
+    for n in (0, 1, 2, 17, 450, 4095):
+        valid = (rng.random(n) < 0.6).astype(np.uint32)
+        speed = np.where(valid == 1, np.round(10.0 ** rng.uniform(-0.7, 1.3, n), 1), 7.0).astype(np.float32)   # many ties
+        fits = _fits(valid, speed)
+        vi = np.nonzero(valid)[0]
+        order = vi[np.lexsort((vi, -speed[vi].astype(np.float64)))]        # speedup descending, then index ascending
+        for k in (1, 4, 10, n + 3):
+            idx, count = oracle.select_elite(fits, k)
+            m = min(k, len(vi))
+            assert count == m and idx[:m].tolist() == order[:m].tolist() and (idx[m:] == 0xFFFFFFFF).all()
+        if len(vi):
+            idx, _ = oracle.select_elite(fits, 1)                           # the single-solution strategy: the best one
+            assert speed[idx[0]] == speed[vi].max() and idx[0] == vi[np.argmax(speed[vi])]
+        # brute force: entry j beats exactly j valid candidates' worth of (speedup, -index) pairs
+        idx, count = oracle.select_elite(fits, n)
+        for j in range(count):
+            i = idx[j]
+            ahead = sum(1 for q in vi if speed[q] > speed[i] or (speed[q] == speed[i] and q < i))
+            assert ahead == j
+    # invalid candidates never appear, whatever their speedup field holds
+    idx, count = oracle.select_elite(_fits([0, 1, 0], [99.0, 0.5, 98.0]), 3)
+    assert count == 1 and idx.tolist() == [1, 0xFFFFFFFF, 0xFFFFFFFF]
