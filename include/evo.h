@@ -252,6 +252,20 @@ EVO_API int evo_summary(evo_ctx* ctx, const evo_fit* fits /* device */, const ui
                         void* stream);
 
 /*
+ * evo_select_elite - which candidates to keep.
+ * Paper: Section 4.2 "Population Management" (the single-solution strategy keeps the current
+ * best solution, elite preservation a small set of high-performing ones).  Writes the indices
+ * of the k valid candidates with the largest speedup, best first, candidates with equal
+ * speedup in order of their index; if fewer than k are valid, the remaining entries are
+ * 0xffffffff.  k = 1 is the single-solution strategy.
+ * fits  : device, n_cand records (as written by evo_fitness); n_cand <= 65536.
+ * idx   : device, k words, written.   count : device, one word: min(k, valid candidates).
+ * Errors: EVO_ERR_ARG, EVO_ERR_ALIGN, EVO_ERR_CUDA.
+ */
+EVO_API int evo_select_elite(evo_ctx* ctx, const evo_fit* fits /* device */, uint64_t n_cand, uint32_t k,
+                             uint32_t* idx /* device */, uint32_t* count /* device */, void* stream);
+
+/*
  * evo_validate_static - evo_validate for callers that cannot allocate device memory.
  * (The paper has no counterpart: this entry point exists for the sake of such callers.)
  *

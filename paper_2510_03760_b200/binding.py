@@ -76,6 +76,8 @@ def load_library():
     L.evo_fitness_ex.restype = i32
     L.evo_summary.argtypes = [vp, vp, vp, vp, u64, u32, u32, vp, vp, vp, vp]
     L.evo_summary.restype = i32
+    L.evo_select_elite.argtypes = [vp, vp, u64, u32, vp, vp, vp]
+    L.evo_select_elite.restype = i32
     _lib = L
     return L
 
@@ -292,6 +294,19 @@ def evo_summary(fits, kernel_of, n_kernel, run_of=None, n_run=1, stream=None, ct
                                     int(n_run), _dev_ptr(out), _dev_ptr(best), _dev_ptr(med), _stream_ptr(stream, dev))
     ctx.check(st)
     return out, best, med
+
+
+def evo_select_elite(fits, k, stream=None, ctx=None):
+    """Indices (int32 CUDA tensor of k entries, -1 where there is none) of the k valid candidates
+    with the largest speedup, best first, and their number (int32 CUDA tensor of one entry)."""
+    dev = fits.device
+    ctx = ctx or default_context(dev.index)
+    idx = torch.empty(int(k), dtype=torch.int32, device=dev)
+    count = torch.empty(1, dtype=torch.int32, device=dev)
+    st = load_library().evo_select_elite(ctx._h, _dev_ptr(fits), fits.shape[0], int(k), _dev_ptr(idx), _dev_ptr(count),
+                                         _stream_ptr(stream, dev))
+    ctx.check(st)
+    return idx, count
 
 
 def summary_to_numpy(summary):

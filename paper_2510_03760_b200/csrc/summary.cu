@@ -126,3 +126,66 @@ extern "C" int evo_summary(evo_ctx* ctx, const evo_fit* fits, const uint32_t* ke
     EVO_CUDA_TRY(ctx, cudaGetLastError());
     return EVO_OK;
 }
+
+// ---- evo_select_elite -----------------------------------------------------------------------
+// Population management (Section 4.2: the single-solution strategy keeps the best candidate,
+// elite preservation a small set of high-performing ones): the k valid candidates with the
+// largest speedup, best first, equal speedups by index.  Rank counting again: a candidate's
+// place is the number of valid candidates ahead of it, so there is no sort and the outcome
+// is unique.  Quadratic in the population, which is a few thousand records.
+namespace {
+
+constexpr uint32_t kMaxEliteCands = 1u << 16;
+constexpr int kEliteThreads = 256;
+
+__global__ void __launch_bounds__(kEliteThreads)
+elite_kernel(const evo_fit* __restrict__ fits, uint32_t n_cand, uint32_t k, uint32_t* __restrict__ idx,
+             uint32_t* __restrict__ count) {
+    __shared__ float s_speed[kEliteThreads];
+    __shared__ uint32_t s_valid[kEliteThreads];
+    const uint32_t i = blockIdx.x * kEliteThreads + threadIdx.x;
+    float mine = 0.f;
+    bool valid = false;
+    if (i < n_cand) { const evo_fit f = fits[i]; mine = f.speedup; valid = f.valid != 0; }
+    uint32_t ahead = 0;
+    for (uint32_t base = 0; base < n_cand; base += kEliteThreads) {
+        const uint32_t j = base + threadIdx.x;
+        __syncthreads();
+        if (j < n_cand) { const evo_fit f = fits[j]; s_speed[threadIdx.x] = f.speedup; s_valid[threadIdx.x] = f.valid; }
+        else s_valid[threadIdx.x] = 0;
+        __syncthreads();
+        const uint32_t lim = min(static_cast<uint32_t>(kEliteThreads), n_cand - base);
+        for (uint32_t q = 0; q < lim; ++q) {
+            const float s = s_speed[q];
+            ahead += (s_valid[q] && (s > mine || (s == mine && base + q < i))) ? 1u : 0u;
+        }
+    }
+    if (valid && ahead < k) {
+        idx[ahead] = i;
+        atomicAdd(count, 1u);           // an integer count: the order of arrival does not matter
+    }
+}
+
+}  // namespace
+
+extern "C" int evo_select_elite(evo_ctx* ctx, const evo_fit* fits, uint64_t n_cand, uint32_t k, uint32_t* idx,
+                                uint32_t* count, void* stream_) {
+    if (!ctx) return EVO_ERR_ARG;
+    const char* who = "evo_select_elite";
+    if (n_cand > kMaxEliteCands) return evo::fail(ctx, EVO_ERR_ARG, "%s: at most %u candidates per call", who, kMaxEliteCands);
+    if (!count || (k > 0 && !idx) || (n_cand > 0 && !fits)) return evo::fail(ctx, EVO_ERR_ARG, "%s: fits, idx and count must not be NULL", who);
+    if (reinterpret_cast<uintptr_t>(fits) % 4 || reinterpret_cast<uintptr_t>(idx) % 4 || reinterpret_cast<uintptr_t>(count) % 4)
+        return evo::fail(ctx, EVO_ERR_ALIGN, "%s: arrays must be 4-byte aligned", who);
+    evo::DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (k > 0) EVO_CUDA_TRY(ctx, cudaMemsetAsync(idx, 0xff, static_cast<size_t>(k) * sizeof(uint32_t), stream));
+    EVO_CUDA_TRY(ctx, cudaMemsetAsync(count, 0, sizeof(uint32_t), stream));
+    if (n_cand > 0 && k > 0) {
+        const unsigned grid = static_cast<unsigned>((n_cand + kEliteThreads - 1) / kEliteThreads);
+        elite_kernel<<<grid, kEliteThreads, 0, stream>>>(fits, static_cast<uint32_t>(n_cand), k, idx, count);
+        ctx->launches += 1;
+        EVO_CUDA_TRY(ctx, cudaGetLastError());
+    }
+    return EVO_OK;
+}

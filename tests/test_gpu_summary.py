@@ -86,3 +86,18 @@ def test_ids_out_of_range_are_reported_and_skipped(evo):
     L = evo.load_library()
     assert L.evo_summary(ctx._h, fits.data_ptr(), fits.data_ptr(), None, 2, 0, 1, fits.data_ptr(), fits.data_ptr(), None, None) == -1
     assert L.evo_summary(ctx._h, fits.data_ptr(), fits.data_ptr(), None, 2, 9000, 1, fits.data_ptr(), fits.data_ptr(), None, None) == -1
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 255, 256, 257, 4095, 20000])
+def test_elite_selection(evo, n):
+    rng = np.random.default_rng(n)
+    valid = (rng.random(n) < 0.6).astype(np.uint32)
+    speed = np.where(valid == 1, np.round(10.0 ** rng.uniform(-0.7, 1.3, n), 1), 7.0).astype(np.float32)   # many ties
+    fits = _fits(valid, speed)
+    d_fits = torch.from_numpy(fits.view(np.uint8).reshape(-1, 16).copy()).cuda() if n else \
+        torch.empty((0, 16), dtype=torch.uint8, device="cuda")
+    for k in (1, 4, 45, n + 3):
+        idx, count = evo.evo_select_elite(d_fits, k)
+        want_idx, want_count = oracle.select_elite(fits, k)
+        assert count.cpu().item() == want_count
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), want_idx)
