@@ -511,3 +511,26 @@ extern "C" int oracle_select_elite(const oracle_fit* fits, uint64_t n_cand, uint
     *count = m;
     return 0;
 }
+
+// ---------------------------------------------------------------------------
+// Feedback on a failing candidate (Section 4.3: the system's third step is
+// feedback collection for the next round of generation): where it is wrong.
+// The first `max_out` elements, in index order, that violate the closeness
+// rule, each with its index and the two values widened to binary32; and the
+// total number of violations.
+// ---------------------------------------------------------------------------
+struct oracle_offender { uint64_t index; float cand; float ref; };
+
+extern "C" int oracle_mismatch_sample(const void* cand, const void* ref, uint64_t n, int dtype, float atol, float rtol,
+                                      uint64_t max_out, oracle_offender* out, uint64_t* n_found) {
+    if (dtype < 1 || dtype > 3) return -1;
+    uint64_t found = 0;
+    for (uint64_t i = 0; i < n; ++i) {
+        const float c = load_widened(cand, i, dtype), r = load_widened(ref, i, dtype);
+        if (!oracle_element_mismatch(c, r, atol, rtol)) continue;
+        if (found < max_out) { out[found].index = i; out[found].cand = c; out[found].ref = r; }
+        ++found;
+    }
+    *n_found = found;
+    return 0;
+}

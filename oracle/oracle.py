@@ -22,6 +22,8 @@ SUMMARY_DTYPE = np.dtype(
      ("hist", "<u4", (5,)), ("n_kernel", "<u4"), ("n_run", "<u4")], align=True)
 assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16 and SUMMARY_DTYPE.itemsize == 48
 STAT_MEDIAN, STAT_MEAN, STAT_MIN, STAT_TRIMMED_MEAN = 0, 1, 2, 3
+OFFENDER_DTYPE = np.dtype([("index", "<u8"), ("cand", "<f4"), ("ref", "<f4")], align=True)
+assert OFFENDER_DTYPE.itemsize == 16
 
 _lib = None
 
@@ -60,6 +62,9 @@ def lib():
         L.oracle_summary.restype = C.c_int
         L.oracle_select_elite.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p]
         L.oracle_select_elite.restype = C.c_int
+        L.oracle_mismatch_sample.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_int, C.c_float, C.c_float, C.c_uint64,
+                                             C.c_void_p, C.c_void_p]
+        L.oracle_mismatch_sample.restype = C.c_int
         _lib = L
     return _lib
 
@@ -217,3 +222,20 @@ def select_elite(fits, k):
     count = np.zeros(1, dtype=np.uint32)
     lib().oracle_select_elite(_ptr(fits), fits.size, int(k), _ptr(idx), _ptr(count))
     return idx, int(count[0])
+
+
+def mismatch_sample(cand, ref, dtype, atol, rtol, max_out):
+    """The first `max_out` elements (index order) that violate the closeness rule, as
+    OFFENDER_DTYPE records, and the total number of violations."""
+    np_dt = np.float32 if dtype == F32 else np.uint16
+    cand = np.ascontiguousarray(cand)
+    ref = np.ascontiguousarray(ref)
+    if cand.dtype != np_dt or ref.dtype != np_dt or cand.size != ref.size:
+        raise TypeError("mismatch_sample: arrays must be %s and of equal size" % np_dt)
+    out = np.zeros(int(max_out), dtype=OFFENDER_DTYPE)
+    found = np.zeros(1, dtype=np.uint64)
+    rc = lib().oracle_mismatch_sample(_ptr(cand), _ptr(ref), cand.size, int(dtype), float(np.float32(atol)),
+                                      float(np.float32(rtol)), int(max_out), _ptr(out), _ptr(found))
+    if rc != 0:
+        raise ValueError("oracle_mismatch_sample: status %d" % rc)
+    return out[: min(int(max_out), int(found[0]))], int(found[0])

@@ -42,6 +42,7 @@
 
 #include "evo_internal.h"
 #include "plan.h"
+#include "rule.cuh"
 
 namespace {
 
@@ -135,39 +136,6 @@ struct Ring {
     __device__ __forceinline__ void advance() { if (++stage == kStages) { stage = 0; phase ^= 1u; } }
 };
 
-// ---- element types ---------------------------------------------------------------------
-template <int DT> struct Elem;
-template <> struct Elem<EVO_F32> {
-    static constexpr int kPerVec = 4;
-    static constexpr int kVecs = kEpt / 4;          // 16-byte vectors per thread per tile
-    using T = float;
-    static __device__ __forceinline__ float at(const uint4& v, int i) {
-        return __uint_as_float(i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w);
-    }
-    static __device__ __forceinline__ float widen(T x) { return x; }
-};
-template <> struct Elem<EVO_F16> {
-    static constexpr int kPerVec = 8;
-    static constexpr int kVecs = kEpt / 8;
-    using T = __half;
-    static __device__ __forceinline__ float at(const uint4& v, int i) {
-        const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
-        const __half2 h = *reinterpret_cast<const __half2*>(&w);
-        return (i & 1) ? __high2float(h) : __low2float(h);
-    }
-    static __device__ __forceinline__ float widen(T x) { return __half2float(x); }
-};
-template <> struct Elem<EVO_BF16> {
-    static constexpr int kPerVec = 8;
-    static constexpr int kVecs = kEpt / 8;
-    using T = __nv_bfloat16;
-    static __device__ __forceinline__ float at(const uint4& v, int i) {
-        const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
-        return __uint_as_float((i & 1) ? (w & 0xffff0000u) : (w << 16));
-    }
-    static __device__ __forceinline__ float widen(T x) { return __bfloat162float(x); }
-};
-
 // ---- the rule, exact form ----------------------------------------------------------------
 // Per-lane state for one (tile, member) on the exact path.
 struct Lane {
@@ -185,10 +153,7 @@ struct Lane {
 __device__ __forceinline__ void exact_elem(float c, float r, float atol, float rtol, Lane& s) {
     const float d = fabsf(__fsub_rn(c, r));
     const float ar = fabsf(r);
-    const float tol = __fadd_rn(atol, __fmul_rn(rtol, ar));
-    const bool d_finite = d < __int_as_float(0x7f800000);          // false for NaN and Inf
-    const bool close = (c == r) || (d_finite && d <= tol);
-    s.cnt += close ? 0u : 1u;
+    s.cnt += rule_mismatch(c, r, atol, rtol) ? 1u : 0u;
     const uint32_t cb = __float_as_uint(c), rb = __float_as_uint(r);
     const uint32_t cm = cb & 0x7fffffffu, rm = rb & 0x7fffffffu;
     uint32_t f = 0;

@@ -1,0 +1,66 @@
+"""Pins for the oracle's offender sample: which elements violate the closeness rule (CPU only)."""
+import numpy as np
+import torch
+
+import oracle
+
+
+def _rule_through_double(c, r, atol, rtol):
+    """The rule with every operation evaluated in binary64 and rounded once to binary32 (53 >= 2*24+2 bits make
+    the double rounding innocuous for +, -, *)."""
+    f = np.float32
+    c, r, atol, rtol = f(c), f(r), f(atol), f(rtol)
+    if c == r:
+        return False
+    with np.errstate(all="ignore"):
+        d = f(abs(np.float64(c) - np.float64(r)))
+        t = f(np.float64(rtol) * abs(np.float64(r)))
+        tol = f(np.float64(atol) + np.float64(t))
+    return not (np.isfinite(d) and d <= tol)
+
+
+def test_sample_against_torch_isclose_and_a_double_precision_loop():
+    rng = np.random.default_rng(3)
+    n = 5000
+    r = rng.standard_normal(n).astype(np.float32)
+    c = (r + 1e-4 * rng.standard_normal(n)).astype(np.float32)
+    bad = rng.choice(n, 40, replace=False)
+    c[bad] = r[bad] + 1.0
+    c[bad[:3]] = [np.nan, np.inf, -np.inf]
+    r[bad[3]] = np.nan
+    c[bad[4]] = r[bad[4]] = np.inf                     # equal infinities match
+    atol = rtol = 0.01
+    close = torch.isclose(torch.from_numpy(c), torch.from_numpy(r), rtol=rtol, atol=atol).numpy()
+    want = np.nonzero(~close)[0]
+    assert len(want) == 39
+    for max_out in (0, 1, 10, 39, 100):
+        got, found = oracle.mismatch_sample(c, r, oracle.F32, atol, rtol, max_out)
+        m = min(max_out, len(want))
+        assert found == len(want) and got["index"].tolist() == want[:m].tolist()
+        assert got["cand"].tobytes() == c[want[:m]].tobytes() and got["ref"].tobytes() == r[want[:m]].tobytes()
+    assert found == oracle.validate(c, r, oracle.F32, atol, rtol)["n_mismatch"]
+    loop = [i for i in range(n) if _rule_through_double(c[i], r[i], atol, rtol)]
+    assert loop == want.tolist()
+
+
+def test_sample_for_sixteen_bit_types_reports_widened_values():
+    rng = np.random.default_rng(4)
+    for dtype in (oracle.F16, oracle.BF16):
+        r32 = rng.standard_normal(3000).astype(np.float32)
+        r = oracle.narrow(dtype, r32)
+        c = oracle.narrow(dtype, r32 + np.where(rng.random(3000) < 0.01, 0.5, 0.0).astype(np.float32))
+        got, found = oracle.mismatch_sample(c, r, dtype, 0.01, 0.01, 1000)
+        cw, rw = oracle.widen(dtype, c), oracle.widen(dtype, r)
+        want = [i for i in range(3000) if _rule_through_double(cw[i], rw[i], 0.01, 0.01)]
+        assert found == len(want) > 5 and got["index"].tolist() == want
+        assert np.array_equal(got["cand"], cw[want]) and np.array_equal(got["ref"], rw[want])
+        assert found == oracle.validate(c, r, dtype, 0.01, 0.01)["n_mismatch"]
+
+
+def test_empty_and_clean_inputs():
+    z = np.zeros(0, np.float32)
+    got, found = oracle.mismatch_sample(z, z, oracle.F32, 0.0, 0.0, 5)
+    assert found == 0 and len(got) == 0
+    x = np.arange(10, dtype=np.float32)
+    got, found = oracle.mismatch_sample(x, x, oracle.F32, 0.0, 0.0, 5)
+    assert found == 0 and len(got) == 0
