@@ -252,6 +252,25 @@ EVO_API int evo_summary(evo_ctx* ctx, const evo_fit* fits /* device */, const ui
                         void* stream);
 
 /*
+ * evo_mismatch_sample - where a failing candidate is wrong.
+ * Paper: Section 4.3 (the third step of the system collects feedback for the next round of
+ * generation).  Judges one candidate tensor against its reference by the rule of evo_validate
+ * and writes the first max_out violating elements in index order: their index and the two
+ * values widened to binary32 (a NaN is reported as some NaN: its payload is not kept);
+ * *n_found receives the total number of violations (so min(max_out, *n_found) entries of
+ * `out` are written; the rest is left untouched).
+ * cand, ref : device, n elements of `dtype` (EVO_F32/F16/BF16), aligned to the element size.
+ * out       : device, max_out entries (may be NULL with max_out 0: count only).
+ * n_found   : device, one 64-bit word.
+ * The context's workspace grows by 8 bytes per 2048 elements.  Errors: EVO_ERR_ARG,
+ * EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_WORKSPACE, EVO_ERR_CUDA.
+ */
+typedef struct { uint64_t index; float cand, ref; } evo_offender;   /* 16 bytes */
+EVO_API int evo_mismatch_sample(evo_ctx* ctx, const void* cand /* device */, const void* ref /* device */, uint64_t n,
+                                int dtype, float atol, float rtol, uint64_t max_out, evo_offender* out /* device */,
+                                uint64_t* n_found /* device */, void* stream);
+
+/*
  * evo_select_elite - which candidates to keep.
  * Paper: Section 4.2 "Population Management" (the single-solution strategy keeps the current
  * best solution, elite preservation a small set of high-performing ones).  Writes the indices

@@ -21,7 +21,8 @@ SUMMARY_DTYPE = np.dtype(
      ("hist", "<u4", (5,)), ("n_kernel", "<u4"), ("n_run", "<u4")], align=True)
 EVO_STAT_MEDIAN, EVO_STAT_MEAN, EVO_STAT_MIN, EVO_STAT_TRIMMED_MEAN = 0, 1, 2, 3
 assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16 and _DESC_DTYPE.itemsize == 24
-assert SUMMARY_DTYPE.itemsize == 48
+OFFENDER_DTYPE = np.dtype([("index", "<u8"), ("cand", "<f4"), ("ref", "<f4")], align=True)
+assert SUMMARY_DTYPE.itemsize == 48 and OFFENDER_DTYPE.itemsize == 16
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libevo.so")
 _lib = None
@@ -78,6 +79,8 @@ def load_library():
     L.evo_summary.restype = i32
     L.evo_select_elite.argtypes = [vp, vp, u64, u32, vp, vp, vp]
     L.evo_select_elite.restype = i32
+    L.evo_mismatch_sample.argtypes = [vp, vp, vp, u64, i32, f32, f32, u64, vp, vp, vp]
+    L.evo_mismatch_sample.restype = i32
     _lib = L
     return L
 
@@ -307,6 +310,27 @@ def evo_select_elite(fits, k, stream=None, ctx=None):
                                          _stream_ptr(stream, dev))
     ctx.check(st)
     return idx, count
+
+
+def evo_mismatch_sample(cand, ref, atol, rtol, max_out, stream=None, ctx=None):
+    """The first `max_out` elements of CUDA tensor `cand` that violate the closeness rule against
+    `ref` (index order).  Returns (numpy OFFENDER_DTYPE records, total number of violations);
+    synchronises to read them back."""
+    if not (cand.is_cuda and ref.is_cuda and cand.is_contiguous() and ref.is_contiguous()):
+        raise ValueError("cand and ref must be contiguous CUDA tensors")
+    if cand.dtype != ref.dtype or cand.numel() != ref.numel():
+        raise ValueError("candidate and reference differ in dtype or size")
+    dev = cand.device
+    ctx = ctx or default_context(dev.index)
+    out = torch.zeros((int(max_out), OFFENDER_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    found = torch.zeros(1, dtype=torch.int64, device=dev)
+    st = load_library().evo_mismatch_sample(ctx._h, _dev_ptr(cand), _dev_ptr(ref), cand.numel(), dtype_code(cand.dtype),
+                                            float(atol), float(rtol), int(max_out), _dev_ptr(out) if max_out else None,
+                                            _dev_ptr(found), _stream_ptr(stream, dev))
+    ctx.check(st)
+    n_found = int(found.cpu().item())
+    recs = out.cpu().numpy().view(OFFENDER_DTYPE).reshape(-1)[: min(int(max_out), n_found)]
+    return recs, n_found
 
 
 def summary_to_numpy(summary):
