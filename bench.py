@@ -363,7 +363,7 @@ def run_ours(args):
 
     cpu = None
     if not args.no_cpu_baseline:
-        sample = OracleSample(args.workload, 27, 25)          # about 10-20 s of single-thread work
+        sample = OracleSample(args.workload, 28, 27)          # about 10-20 s of single-thread work
         est, spent = sample.run()
         cpu = {"value": alg_bytes / est / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.description,
                "seconds": spent, "host_cores_available": os.cpu_count()}

@@ -29,3 +29,56 @@ def test_config4_full_size():
     wrong = pop.facts["wrong"]
     assert got["pass"].sum() == 15 and got["pass"][wrong] == 0 and got["n_mismatch"][wrong] > 0.99 * (1 << 28)
     assert gp.cpu().tolist() == got["pass"].tolist()
+
+
+def test_config3_full_size():
+    """128 candidates x 2^20 fp16/bf16 elements with NaN/Inf and boundary values: every tensor by the oracle."""
+    import paper_2510_03760_b200 as evo
+    pop = workloads.config3("cuda")
+    cands = [t.cand for t in pop.tensors]
+    refs = [pop.refs[t.ref_index] for t in pop.tensors]
+    groups = [t.group for t in pop.tensors]
+    res, gp = evo.evo_validate(cands, refs, pop.atol, pop.rtol, groups=groups, n_group=pop.n_group)
+    got = evo.results_to_numpy(res)
+    host_refs = [workloads.to_host_bits(r) for r in pop.refs]
+    want = np.zeros(len(cands), dtype=oracle.RESULT_DTYPE)
+    for i, t in enumerate(pop.tensors):
+        want[i] = oracle.validate(workloads.to_host_bits(t.cand), host_refs[t.ref_index], t.dtype, pop.atol, pop.rtol)
+    assert_results_equal(got, want, "config3 full size")
+    assert want["n_nonfinite"].sum() > 50 and (want["flags"] != 0).sum() > 30        # the specials are really there
+    assert np.array_equal(gp.cpu().numpy().view(np.uint32), oracle.group_pass(want, groups, pop.n_group))
+
+
+def test_config5_full_size_sampled():
+    """The ragged population at full size (1024 candidates, about 2000 tensors, 22 GB): a seeded sample of tensors
+    by the oracle element by element, and for all of them what holds by construction."""
+    import paper_2510_03760_b200 as evo
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * (1 << 30):
+        pytest.skip("needs 60 GiB of device memory")
+    pop = workloads.config5("cuda")
+    cands = [t.cand for t in pop.tensors]
+    refs = [pop.refs[t.ref_index] for t in pop.tensors]
+    groups = [t.group for t in pop.tensors]
+    res, gp = evo.evo_validate(cands, refs, pop.atol, pop.rtol, groups=groups, n_group=pop.n_group)
+    got = evo.results_to_numpy(res)
+    gp = gp.cpu().numpy()
+    # by construction: candidates without injected elements pass; no NaN/Inf anywhere; errors below the tolerance scale
+    rates = pop.facts["rates"]
+    for i, t in enumerate(pop.tensors):
+        if rates[t.group] == 0.0:
+            assert got["pass"][i] == 1 and got["n_mismatch"][i] == 0, i
+        assert got["n_nonfinite"][i] == 0 and got["flags"][i] == 0
+        assert got["n_mismatch"][i] <= t.cand.numel()
+    for g in range(pop.n_group):
+        mine = [i for i, t in enumerate(pop.tensors) if t.group == g]
+        assert gp[g] == int(all(got["pass"][i] for i in mine))
+    # a seeded sample, biased to cover the largest and the smallest tensors and every dtype
+    rng = np.random.default_rng(55)
+    order = np.argsort([t.cand.numel() for t in pop.tensors])
+    sample = set(order[:8].tolist()) | set(order[-6:].tolist()) | set(rng.choice(len(cands), 40, replace=False).tolist())
+    for i in sorted(sample):
+        t = pop.tensors[i]
+        want = oracle.validate(workloads.to_host_bits(t.cand), workloads.to_host_bits(pop.refs[t.ref_index]), t.dtype,
+                               pop.atol, pop.rtol)
+        assert_results_equal(got[i:i + 1], np.array([want]), "config5 tensor %d (n=%d, dtype=%d)" % (i, t.cand.numel(), t.dtype))
