@@ -534,3 +534,45 @@ extern "C" int oracle_mismatch_sample(const void* cand, const void* ref, uint64_
     *n_found = found;
     return 0;
 }
+
+// ---------------------------------------------------------------------------
+// Integer and boolean outputs (index results such as an argmax, masks, counts).
+// The paper's constraint is that the output matches the reference (Section 3.1,
+// Eq. 1; Section 4.3); for these types that is read as equality, element by
+// element.  Reports the number of unequal elements and the largest |c - r|,
+// exactly, as an unsigned 64-bit integer.  dtype: 5 = int32, 6 = int64,
+// 7 = uint8 (also bool).
+// ---------------------------------------------------------------------------
+struct oracle_result_exact { uint64_t n_mismatch; uint64_t max_abs_diff; uint32_t pass; uint32_t pad; };
+
+extern "C" int oracle_validate_exact(const void* cand, const void* ref, uint64_t n, int dtype, oracle_result_exact* out) {
+    oracle_result_exact res{};
+    for (uint64_t i = 0; i < n; ++i) {
+        uint64_t diff;
+        if (dtype == 5) {
+            const int64_t c = static_cast<const int32_t*>(cand)[i], r = static_cast<const int32_t*>(ref)[i];
+            diff = static_cast<uint64_t>(c > r ? c - r : r - c);
+        } else if (dtype == 6) {
+            const int64_t c = static_cast<const int64_t*>(cand)[i], r = static_cast<const int64_t*>(ref)[i];
+            // the true difference may not fit int64: subtract as unsigned (exact modulo 2^64, and below 2^64)
+            diff = c > r ? static_cast<uint64_t>(c) - static_cast<uint64_t>(r) : static_cast<uint64_t>(r) - static_cast<uint64_t>(c);
+        } else if (dtype == 7) {
+            const int c = static_cast<const uint8_t*>(cand)[i], r = static_cast<const uint8_t*>(ref)[i];
+            diff = static_cast<uint64_t>(c > r ? c - r : r - c);
+        } else {
+            return -1;
+        }
+        if (diff != 0) ++res.n_mismatch;
+        if (diff > res.max_abs_diff) res.max_abs_diff = diff;
+    }
+    res.pass = res.n_mismatch == 0 ? 1u : 0u;
+    *out = res;
+    return 0;
+}
+
+extern "C" void oracle_group_pass_exact(const oracle_result_exact* results, const uint32_t* group, uint64_t n_desc,
+                                        uint32_t* group_pass, uint64_t n_group) {
+    for (uint64_t g = 0; g < n_group; ++g) group_pass[g] = 1u;
+    for (uint64_t i = 0; i < n_desc; ++i)
+        if (group[i] < n_group && !results[i].pass) group_pass[group[i]] = 0u;
+}

@@ -22,6 +22,10 @@ SUMMARY_DTYPE = np.dtype(
      ("hist", "<u4", (5,)), ("n_kernel", "<u4"), ("n_run", "<u4")], align=True)
 assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16 and SUMMARY_DTYPE.itemsize == 48
 STAT_MEDIAN, STAT_MEAN, STAT_MIN, STAT_TRIMMED_MEAN = 0, 1, 2, 3
+I32, I64, U8 = 5, 6, 7
+_EXACT_NP = {I32: np.int32, I64: np.int64, U8: np.uint8}
+EXACT_DTYPE = np.dtype([("n_mismatch", "<u8"), ("max_abs_diff", "<u8"), ("pass", "<u4"), ("pad", "<u4")], align=True)
+assert EXACT_DTYPE.itemsize == 24
 OFFENDER_DTYPE = np.dtype([("index", "<u8"), ("cand", "<f4"), ("ref", "<f4")], align=True)
 assert OFFENDER_DTYPE.itemsize == 16
 
@@ -65,6 +69,10 @@ def lib():
         L.oracle_mismatch_sample.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_int, C.c_float, C.c_float, C.c_uint64,
                                              C.c_void_p, C.c_void_p]
         L.oracle_mismatch_sample.restype = C.c_int
+        L.oracle_validate_exact.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_int, C.c_void_p]
+        L.oracle_validate_exact.restype = C.c_int
+        L.oracle_group_pass_exact.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64]
+        L.oracle_group_pass_exact.restype = None
         _lib = L
     return _lib
 
@@ -239,3 +247,27 @@ def mismatch_sample(cand, ref, dtype, atol, rtol, max_out):
     if rc != 0:
         raise ValueError("oracle_mismatch_sample: status %d" % rc)
     return out[: min(int(max_out), int(found[0]))], int(found[0])
+
+
+def validate_exact(cand, ref, dtype):
+    """Integer / boolean tensors: equality, element by element.  Returns an EXACT_DTYPE scalar."""
+    np_dt = _EXACT_NP[dtype]
+    cand = np.ascontiguousarray(cand)
+    ref = np.ascontiguousarray(ref)
+    if cand.dtype == np.bool_:
+        cand, ref = cand.view(np.uint8), ref.view(np.uint8)
+    if cand.dtype != np_dt or ref.dtype != np_dt or cand.size != ref.size:
+        raise TypeError("validate_exact: arrays must be %s and of equal size" % np_dt)
+    out = np.zeros(1, dtype=EXACT_DTYPE)
+    rc = lib().oracle_validate_exact(_ptr(cand), _ptr(ref), cand.size, int(dtype), _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_validate_exact: status %d" % rc)
+    return out[0]
+
+
+def group_pass_exact(results, group, n_group):
+    results = np.ascontiguousarray(results, dtype=EXACT_DTYPE)
+    group = np.ascontiguousarray(group, dtype=np.uint32)
+    out = np.empty(int(n_group), dtype=np.uint32)
+    lib().oracle_group_pass_exact(_ptr(results), _ptr(group), results.size, _ptr(out), int(n_group))
+    return out

@@ -64,3 +64,29 @@ def test_empty_and_clean_inputs():
     x = np.arange(10, dtype=np.float32)
     got, found = oracle.mismatch_sample(x, x, oracle.F32, 0.0, 0.0, 5)
     assert found == 0 and len(got) == 0
+
+
+def test_integer_outputs_against_numpy_and_unbounded_integers():
+    rng = np.random.default_rng(9)
+    cases = [
+        (oracle.I32, rng.integers(-2**31, 2**31, 5000, dtype=np.int64).astype(np.int32)),
+        (oracle.I64, rng.integers(-2**63, 2**63 - 1, 5000, dtype=np.int64)),
+        (oracle.U8, rng.integers(0, 256, 5000, dtype=np.int64).astype(np.uint8)),
+    ]
+    for dtype, r in cases:
+        c = r.copy()
+        res = oracle.validate_exact(c, r, dtype)
+        assert res["n_mismatch"] == 0 and res["max_abs_diff"] == 0 and res["pass"] == 1
+        idx = rng.choice(r.size, 37, replace=False)
+        c[idx] = np.roll(r, 1)[idx]                       # some of these may coincide by chance
+        info = np.iinfo(r.dtype)
+        c[0], r[0] = info.max, info.min                    # the widest possible difference
+        res = oracle.validate_exact(c, r, dtype)
+        assert res["n_mismatch"] == np.count_nonzero(c != r) > 30 and res["pass"] == 0
+        assert int(res["max_abs_diff"]) == max(abs(int(a) - int(b)) for a, b in zip(c, r)) == int(info.max) - int(info.min)
+    b = rng.random(1000) < 0.5
+    res = oracle.validate_exact(b, ~b, oracle.U8)
+    assert res["n_mismatch"] == 1000 and res["max_abs_diff"] == 1
+    assert oracle.validate_exact(np.zeros(0, np.int32), np.zeros(0, np.int32), oracle.I32)["pass"] == 1
+    gp = oracle.group_pass_exact(np.array([(0, 0, 1, 0), (3, 9, 0, 0), (0, 0, 1, 0)], oracle.EXACT_DTYPE), [0, 0, 2], 3)
+    assert gp.tolist() == [0, 1, 1]
