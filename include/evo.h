@@ -60,8 +60,9 @@ enum {
     EVO_ERR_TIMEOUT = -6     /* a bounded device-side wait gave up (reported through the context status word) */
 };
 
-/* Element types. EVO_U32 is accepted by evo_gen_inputs only. */
-enum { EVO_U32 = 0, EVO_F32 = 1, EVO_F16 = 2, EVO_BF16 = 3 };
+/* Element types. EVO_U32 is accepted by evo_gen_inputs only; EVO_I32, EVO_I64 and EVO_U8 (also
+ * the storage of bool) by evo_validate_exact only. */
+enum { EVO_U32 = 0, EVO_F32 = 1, EVO_F16 = 2, EVO_BF16 = 3, EVO_I32 = 5, EVO_I64 = 6, EVO_U8 = 7 };
 
 /* Bits of evo_result.flags. */
 enum {
@@ -250,6 +251,23 @@ EVO_API int evo_summary(evo_ctx* ctx, const evo_fit* fits /* device */, const ui
                         const uint32_t* run_of /* device, optional */, uint64_t n_cand, uint32_t n_kernel, uint32_t n_run,
                         evo_summary_rec* out /* device */, float* best /* device */, float* run_median /* device, optional */,
                         void* stream);
+
+/*
+ * evo_validate_exact - the correctness constraint for integer and boolean outputs (index
+ * results such as an argmax, masks, counts).
+ * Paper: Section 3.1 Eq. 1 and Section 4.3 (the output must match the reference); for these
+ * types "match" is read as equality, element by element.  Arguments as evo_validate, without
+ * tolerances; descriptor and call dtypes are EVO_I32, EVO_I64 or EVO_U8.  Per tensor it
+ * reports the number of unequal elements and the largest |c - r| (exact, as an unsigned
+ * 64-bit integer: the difference of two int64 values always fits); pass = (n_mismatch == 0).
+ * Tensors that share (reference, n, dtype) are found and their reference is read once.
+ * Errors: EVO_ERR_ARG, EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_WORKSPACE, EVO_ERR_CUDA.
+ */
+typedef struct { uint64_t n_mismatch; uint64_t max_abs_diff; uint32_t pass; uint32_t pad; } evo_result_exact;   /* 24 bytes */
+EVO_API int evo_validate_exact(evo_ctx* ctx, const void* const* cand_ptrs /* host array of device ptrs */,
+                               const void* ref_ptr /* device */, const evo_desc* descs /* host */, uint64_t n_desc, int dtype,
+                               evo_result_exact* results /* device */, uint32_t* group_pass /* device, optional */,
+                               uint64_t n_group, void* stream);
 
 /*
  * evo_mismatch_sample - where a failing candidate is wrong.

@@ -40,7 +40,7 @@ int plan_fail(std::string* err, int status, const char* fmt, ...) {
 
 int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs, uint64_t n_desc,
                int dtype, float atol, float rtol, bool want_groups, uint64_t n_group, uint32_t max_ctas,
-               Plan* plan, std::string* err) {
+               Plan* plan, std::string* err, uint32_t accepted_types) {
     if (!(atol >= 0.f) || !(rtol >= 0.f) || std::isinf(atol) || std::isinf(rtol))
         return plan_fail(err, EVO_ERR_ARG, "atol and rtol must be finite and >= 0");
     if (want_groups != (n_group != 0)) return plan_fail(err, EVO_ERR_ARG, "group_pass and n_group must be given together");
@@ -57,12 +57,12 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
         const evo_desc& d = descs[i];
         const int dt = d.dtype == -1 ? dtype : d.dtype;
         const unsigned long long ii = i;
-        if (dt != EVO_F32 && dt != EVO_F16 && dt != EVO_BF16)
+        if (dt < 0 || dt > 31 || !((accepted_types >> dt) & 1u) || dtype_bytes(dt) == 0)
             return plan_fail(err, EVO_ERR_DTYPE, "descriptor %llu has dtype %d", ii, dt);
         const void* ref = d.ref ? d.ref : ref_ptr;
         if (d.n > 0 && (!ref || !cand_ptrs[i])) return plan_fail(err, EVO_ERR_ARG, "descriptor %llu has a NULL tensor", ii);
         if (d.n > (1ull << 60)) return plan_fail(err, EVO_ERR_ARG, "descriptor %llu is too large", ii);
-        const size_t eb = dt == EVO_F32 ? 4 : 2;
+        const size_t eb = dtype_bytes(dt);
         if (d.n > 0 && (reinterpret_cast<uintptr_t>(ref) % eb || reinterpret_cast<uintptr_t>(cand_ptrs[i]) % eb))
             return plan_fail(err, EVO_ERR_ALIGN, "descriptor %llu is not aligned to %zu bytes", ii, eb);
         if (want_groups && d.group >= n_group)

@@ -55,6 +55,19 @@ struct CtaRange {            // items [(s_begin, t_begin), (s_end, t_end)) with 
     uint32_t first_member;   // member_off of s_begin
 };
 
+// Bytes per element of every type a plan can hold (0: not a type).
+inline uint32_t dtype_bytes(int dt) {
+    switch (dt) {
+        case EVO_F32: case EVO_I32: return 4;
+        case EVO_F16: case EVO_BF16: return 2;
+        case EVO_I64: return 8;
+        case EVO_U8: return 1;
+        default: return 0;
+    }
+}
+constexpr uint32_t kFloatTypes = (1u << EVO_F32) | (1u << EVO_F16) | (1u << EVO_BF16);
+constexpr uint32_t kIntTypes = (1u << EVO_I32) | (1u << EVO_I64) | (1u << EVO_U8);
+
 struct Plan {
     std::vector<SetRec> sets;
     std::vector<MemberRec> members;      // ordered by set
@@ -69,6 +82,6 @@ struct Plan {
 // Pure host code (no CUDA call).  Returns EVO_OK or an EVO_ERR_* with `err` set.
 int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs, uint64_t n_desc,
                int dtype, float atol, float rtol, bool want_groups, uint64_t n_group, uint32_t max_ctas,
-               Plan* plan, std::string* err);
+               Plan* plan, std::string* err, uint32_t accepted_types = kFloatTypes);
 
 }  // namespace evo
