@@ -134,6 +134,7 @@ int evo_destroy(evo_ctx* ctx) {
     if (ctx->d_partials) (void)cudaFree(ctx->d_partials);
     if (ctx->d_stage) (void)cudaFree(ctx->d_stage);
     if (ctx->d_feedback) (void)cudaFree(ctx->d_feedback);
+    if (ctx->d_seeds) (void)cudaFree(ctx->d_seeds);
     if (ctx->d_small) (void)cudaFree(ctx->d_small);
     if (ctx->plan_consumed) (void)cudaEventDestroy(ctx->plan_consumed);
     delete ctx;

@@ -53,6 +53,7 @@ constexpr int kStages = 6;                          // ring depth per CTA
 constexpr int kStageBytes = kTileElems * 4;         // 16 KiB: one fp32 tile (a 16-bit tile uses half)
 constexpr size_t kRingBytes = static_cast<size_t>(kStages) * kStageBytes;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, then give up
+constexpr uint64_t kSeedBelowTilesPerCta = 32;               // runs shorter than this get the seed pass
 
 // ---- shared-memory barriers and bulk copies (PTX) -------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -565,7 +566,7 @@ __device__ __forceinline__ uint32_t producer_loop(const SetRec* __restrict__ set
 __global__ void __launch_bounds__(kBlock, kCtasPerSm)
 validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
                const CtaRange* __restrict__ ranges, Acc* __restrict__ partials, float atol, float rtol,
-               uint32_t* __restrict__ status) {
+               uint32_t* __restrict__ status, const uint32_t* __restrict__ seeds /* optional: see seed_kernel */) {
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ Acc s_acc[kMaxK][kWarps];
     __shared__ const void* s_cand[kMaxK];
@@ -604,7 +605,7 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
             }
             if (threadIdx.x < S.k) {
                 s_cand[threadIdx.x] = members[S.member_off + threadIdx.x].cand;
-                s_mr[threadIdx.x] = 0;
+                s_mr[threadIdx.x] = seeds ? seeds[S.member_off + threadIdx.x] : 0u;
             }
             consumer_bar();
             if (S.dtype == EVO_F32) run_set<EVO_F32>(S, sp, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
@@ -640,6 +641,39 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
             }
         }
         if (threadIdx.x == 0) atomicOr(status, 1u);
+    }
+}
+
+// Warm start for the filter of max d/|r|.  A CTA that begins a run knows no maximum for its
+// members yet, so on its first tile every lane's filter fires and the exact handling runs for
+// the whole tile; with short runs (a few tiles per CTA and member) that is a large share of the
+// work.  This small kernel, run before the first pass when runs are short, takes the exact
+// maximum quotient over the first tile of every member (one CTA per member, a division per
+// element) and the first pass starts every run from it.  The seed is a true quotient of that
+// member, so folding it into the result changes nothing: the maximum is the maximum.
+__global__ void __launch_bounds__(kThreads)
+seed_kernel(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members, uint32_t* __restrict__ seeds) {
+    __shared__ uint32_t s_max[kWarps];
+    const MemberRec M = members[blockIdx.x];
+    const SetRec S = sets[M.set];
+    const uint64_t n = S.n < static_cast<uint64_t>(kTileElems) ? S.n : static_cast<uint64_t>(kTileElems);
+    float best = 0.f;
+    for (uint64_t e = threadIdx.x; e < n; e += kThreads) {
+        float c, r;
+        if (S.dtype == EVO_F32) { c = static_cast<const float*>(M.cand)[e]; r = static_cast<const float*>(S.ref)[e]; }
+        else if (S.dtype == EVO_F16) { c = __half2float(static_cast<const __half*>(M.cand)[e]); r = __half2float(static_cast<const __half*>(S.ref)[e]); }
+        else { c = __bfloat162float(static_cast<const __nv_bfloat16*>(M.cand)[e]); r = __bfloat162float(static_cast<const __nv_bfloat16*>(S.ref)[e]); }
+        const float d = fabsf(__fsub_rn(c, r)), ar = fabsf(r);
+        const bool usable = d > 0.f && ar > 0.f && d < kInf && ar < kInf && fabsf(c) < kInf;      // as the statistics: finite pairs, r != 0
+        if (usable) best = fmaxf(best, __fdiv_rn(d, ar));
+    }
+    const uint32_t w = __reduce_max_sync(0xffffffffu, __float_as_uint(best));
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = w;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t m = 0;
+        for (int i = 0; i < kWarps; ++i) m = max(m, s_max[i]);
+        seeds[blockIdx.x] = m;
     }
 }
 
@@ -753,6 +787,14 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     if (st != EVO_OK) return st;
     st = evo::reserve_device(ctx, &ctx->d_partials, &ctx->d_partials_bytes, std::max<size_t>(plan.n_parts, 1) * sizeof(Acc));
     if (st != EVO_OK) return st;
+    // Short runs (few tiles per CTA and member): seed the filter of max d/|r| first, see seed_kernel.
+    // (Not for populations with fewer tiles than CTAs: those are bound by launch latency, which a further
+    // kernel only adds to.)
+    const bool seed = plan.total_tiles >= max_ctas && plan.total_tiles / max_ctas < kSeedBelowTilesPerCta;
+    if (seed) {
+        st = evo::reserve_device(ctx, &ctx->d_seeds, &ctx->d_seeds_bytes, std::max<size_t>(n_desc, 1) * sizeof(uint32_t));
+        if (st != EVO_OK) return st;
+    }
     if (ctx->plan_in_flight) {
         // the pinned staging block is about to be overwritten: the previous upload must have been read
         EVO_CUDA_TRY(ctx, cudaEventSynchronize(ctx->plan_consumed));
@@ -780,13 +822,21 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     ctx->time_start = ctx->time_stop = nullptr;
     if (ev_start) EVO_CUDA_TRY(ctx, cudaEventRecord(ev_start, stream));
     uint32_t* d_status = evo::status_word(ctx);
+    const uint32_t* d_seeds = nullptr;
+    if (seed && n_desc > 0) {
+        seed_kernel<<<static_cast<unsigned>(n_desc), kThreads, 0, stream>>>(d_sets, d_members, static_cast<uint32_t*>(ctx->d_seeds));
+        ctx->launches += 1;
+        EVO_CUDA_TRY(ctx, cudaGetLastError());
+        d_seeds = static_cast<const uint32_t*>(ctx->d_seeds);
+    }
     if (n_ctas > 0) {
         if (!ctx->pass1_ready) {
             EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(validate_pass1, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    static_cast<int>(kRingBytes)));
             ctx->pass1_ready = true;
         }
-        validate_pass1<<<n_ctas, kBlock, kRingBytes, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol, d_status);
+        validate_pass1<<<n_ctas, kBlock, kRingBytes, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol, d_status,
+                                                               d_seeds);
         ctx->launches += 1;
         EVO_CUDA_TRY(ctx, cudaGetLastError());
     }
@@ -1008,7 +1058,8 @@ extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref
     uint32_t* d_status = reinterpret_cast<uint32_t*>(dev.scratch);
     const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
     if (n_ctas > 0)
-        validate_pass1<<<n_ctas, kBlock, kRingBytes, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol, d_status);
+        validate_pass1<<<n_ctas, kBlock, kRingBytes, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol, d_status,
+                                                               nullptr);
     const uint32_t n_members = static_cast<uint32_t>(n_desc);
     if (n_members > 0)
         validate_pass2<<<(n_members + kWarps - 1) / kWarps, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts,
