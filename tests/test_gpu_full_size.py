@@ -82,3 +82,46 @@ def test_config5_full_size_sampled():
         want = oracle.validate(workloads.to_host_bits(t.cand), workloads.to_host_bits(pop.refs[t.ref_index]), t.dtype,
                                pop.atol, pop.rtol)
         assert_results_equal(got[i:i + 1], np.array([want]), "config5 tensor %d (n=%d, dtype=%d)" % (i, t.cand.numel(), t.dtype))
+
+
+def test_tensor_beyond_2_to_32_elements():
+    """One bf16 tensor of 2^32 + 12293 elements (8 GiB each for candidate and reference): indices and counts past
+    32 bits.  The candidate equals the reference except at planted positions around 2^31, 2^32 and the very end, so
+    every statistic is known by construction; windows around the planted positions also go through the oracle."""
+    import paper_2510_03760_b200 as evo
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * (1 << 30):
+        pytest.skip("needs 40 GiB of device memory")
+    n = (1 << 32) + 3 * 4096 + 5
+    g = torch.Generator(device="cuda").manual_seed(99)
+    ref = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    step = 1 << 28
+    for lo in range(0, n, step):                                   # in slices: the generator's fp32 temporaries stay small
+        hi = min(n, lo + step)
+        ref[lo:hi] = torch.randn(hi - lo, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    cand = ref.clone()
+    planted = [0, 4095, (1 << 31) - 1, 1 << 31, (1 << 32) - 1, 1 << 32, (1 << 32) + 4096, n - 6, n - 1]
+    for p in planted:
+        cand[p] = ref[p].float() + 1.0
+    nan_at = (1 << 32) + 7
+    cand[nan_at] = float("nan")
+    atol = rtol = 0.01
+    res, _ = evo.evo_validate([cand], [ref], atol, rtol)
+    got = evo.results_to_numpy(res)[0]
+    d = np.array([abs(np.float32(cand[p].float().item()) - np.float32(ref[p].float().item())) for p in planted], np.float32)
+    rr = np.array([abs(np.float32(ref[p].float().item())) for p in planted], np.float32)
+    assert (d > np.float32(atol) + np.float32(rtol) * rr).all()
+    assert got["n_mismatch"] == len(planted) + 1 and got["n_nonfinite"] == 1 and got["flags"] == 1 and got["pass"] == 0
+    assert got["max_abs"] == d.max() and got["max_rel"] == (d / rr).max()
+    want_sse = float(np.sum(d.astype(np.float64) ** 2))
+    assert abs(got["sse"] - want_sse) <= 1e-5 * want_sse
+    # the offenders, with 64-bit indices
+    recs, found = evo.evo_mismatch_sample(cand, ref, atol, rtol, 64)
+    assert found == len(planted) + 1
+    assert recs["index"].tolist() == sorted(planted + [nan_at])
+    # windows around the planted positions through the oracle
+    for p in (1 << 31, 1 << 32, n - 1):
+        lo, hi = max(0, p - 5000), min(n, p + 5000)
+        w_res, _ = evo.evo_validate([cand[lo:hi]], [ref[lo:hi]], atol, rtol)
+        want = oracle.validate(workloads.to_host_bits(cand[lo:hi]), workloads.to_host_bits(ref[lo:hi]), oracle.BF16, atol, rtol)
+        assert_results_equal(evo.results_to_numpy(w_res), np.array([want]), "window at %d" % p)
