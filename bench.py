@@ -308,7 +308,8 @@ def run_ours(args):
     if not args.no_e2e:
         import psutil
         need = alg_bytes + (2 << 30)
-        if psutil.virtual_memory().available > 2 * need and torch.cuda.mem_get_info()[0] > need:
+        # every rank of the node pins its own copy at the same time: budget the host memory for all of them
+        if psutil.virtual_memory().available > 2 * need * world and torch.cuda.mem_get_info()[0] > need:
             h_refs = [r.cpu().pin_memory() for r in pop.refs]
             h_cands = [t.cand.cpu().pin_memory() for t in pop.tensors]
             aliasing = False
