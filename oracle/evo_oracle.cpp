@@ -576,3 +576,44 @@ extern "C" void oracle_group_pass_exact(const oracle_result_exact* results, cons
     for (uint64_t i = 0; i < n_desc; ++i)
         if (group[i] < n_group && !results[i].pass) group_pass[group[i]] = 0u;
 }
+
+// ---------------------------------------------------------------------------
+// binary64 outputs: the same rule and statistics as oracle_validate, with every
+// operation an individually rounded binary64 operation (no fused multiply-add):
+// d = |c - r|, tol = atol + rtol*|r|, close = (c == r) or (d finite and d <= tol);
+// NaN/Inf elements are counted and flagged and stay out of max_abs, max_rel and
+// sse.  The sum of squares is accumulated in extended precision (long double) so
+// that the oracle's own summation error stays far below the comparison bar.
+// ---------------------------------------------------------------------------
+struct oracle_result64 {
+    uint64_t n_mismatch, n_nonfinite;
+    double sse, max_abs, max_rel;
+    uint32_t flags, pass;
+};
+
+extern "C" int oracle_validate_f64(const double* cand, const double* ref, uint64_t n, double atol, double rtol,
+                                   oracle_result64* out) {
+    oracle_result64 res{};
+    long double sse = 0.0L;
+    for (uint64_t i = 0; i < n; ++i) {
+        const double c = cand[i], r = ref[i];
+        const double d = std::fabs(c - r);
+        const double t = rtol * std::fabs(r);
+        const double tol = atol + t;
+        const bool close = (c == r) || (std::isfinite(d) && d <= tol);
+        if (!close) ++res.n_mismatch;
+        uint32_t f = 0;
+        if (std::isnan(c)) f |= 1u;
+        if (std::isinf(c)) f |= (c > 0 ? 2u : 4u);
+        if (std::isnan(r)) f |= 8u;
+        if (std::isinf(r)) f |= 16u;
+        if (f) { ++res.n_nonfinite; res.flags |= f; continue; }
+        if (d > res.max_abs) res.max_abs = d;
+        if (r != 0.0) { const double q = d / std::fabs(r); if (q > res.max_rel) res.max_rel = q; }
+        sse += static_cast<long double>(d) * static_cast<long double>(d);
+    }
+    res.sse = static_cast<double>(sse);
+    res.pass = res.n_mismatch == 0 ? 1u : 0u;
+    *out = res;
+    return 0;
+}

@@ -26,6 +26,10 @@ I32, I64, U8 = 5, 6, 7
 _EXACT_NP = {I32: np.int32, I64: np.int64, U8: np.uint8}
 EXACT_DTYPE = np.dtype([("n_mismatch", "<u8"), ("max_abs_diff", "<u8"), ("pass", "<u4"), ("pad", "<u4")], align=True)
 assert EXACT_DTYPE.itemsize == 24
+RESULT64_DTYPE = np.dtype(
+    [("n_mismatch", "<u8"), ("n_nonfinite", "<u8"), ("sse", "<f8"), ("max_abs", "<f8"), ("max_rel", "<f8"),
+     ("flags", "<u4"), ("pass", "<u4")], align=True)
+assert RESULT64_DTYPE.itemsize == 48
 OFFENDER_DTYPE = np.dtype([("index", "<u8"), ("cand", "<f4"), ("ref", "<f4")], align=True)
 assert OFFENDER_DTYPE.itemsize == 16
 
@@ -73,6 +77,8 @@ def lib():
         L.oracle_validate_exact.restype = C.c_int
         L.oracle_group_pass_exact.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64]
         L.oracle_group_pass_exact.restype = None
+        L.oracle_validate_f64.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_double, C.c_double, C.c_void_p]
+        L.oracle_validate_f64.restype = C.c_int
         _lib = L
     return _lib
 
@@ -271,3 +277,16 @@ def group_pass_exact(results, group, n_group):
     out = np.empty(int(n_group), dtype=np.uint32)
     lib().oracle_group_pass_exact(_ptr(results), _ptr(group), results.size, _ptr(out), int(n_group))
     return out
+
+
+def validate_f64(cand, ref, atol, rtol):
+    """binary64 tensors: the rule and statistics in binary64.  Returns a RESULT64_DTYPE scalar."""
+    cand = np.ascontiguousarray(cand)
+    ref = np.ascontiguousarray(ref)
+    if cand.dtype != np.float64 or ref.dtype != np.float64 or cand.size != ref.size:
+        raise TypeError("validate_f64: arrays must be float64 and of equal size")
+    out = np.zeros(1, dtype=RESULT64_DTYPE)
+    rc = lib().oracle_validate_f64(_ptr(cand), _ptr(ref), cand.size, float(atol), float(rtol), _ptr(out))
+    if rc != 0:
+        raise ValueError("oracle_validate_f64: status %d" % rc)
+    return out[0]

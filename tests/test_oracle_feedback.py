@@ -90,3 +90,59 @@ def test_integer_outputs_against_numpy_and_unbounded_integers():
     assert oracle.validate_exact(np.zeros(0, np.int32), np.zeros(0, np.int32), oracle.I32)["pass"] == 1
     gp = oracle.group_pass_exact(np.array([(0, 0, 1, 0), (3, 9, 0, 0), (0, 0, 1, 0)], oracle.EXACT_DTYPE), [0, 0, 2], 3)
     assert gp.tolist() == [0, 1, 1]
+
+
+def test_binary64_rule_against_numpy_isclose_exact_rationals_and_fsum():
+    import math
+    from fractions import Fraction
+    rng = np.random.default_rng(12)
+    n = 20000
+    r = rng.standard_normal(n)
+    c = r + 1e-9 * rng.standard_normal(n)
+    atol, rtol = 1e-8, 1e-8
+    # values right at the boundary, decided with exact rationals applied to the individually rounded operations
+    tol = atol + rtol * np.abs(r)                      # numpy: one binary64 rounding per operation, as the rule says
+    for i, ulps in zip(range(0, 600, 3), np.tile([-1, 0, 1], 200)):
+        c[i] = r[i] + tol[i]
+        for _ in range(abs(int(ulps))):
+            c[i] = np.nextafter(c[i], np.inf if ulps > 0 else -np.inf)
+    special = rng.choice(np.arange(1000, n), 12, replace=False)
+    c[special[:3]] = [np.nan, np.inf, -np.inf]
+    r[special[3]] = np.nan
+    c[special[4]] = r[special[4]] = np.inf
+    r[special[5]] = 0.0
+    c[special[6]], r[special[6]] = 1e308, -1e308        # the difference overflows
+    res = oracle.validate_f64(c, r, atol, rtol)
+    with np.errstate(all="ignore"):
+        close = np.isclose(c, r, rtol=rtol, atol=atol)
+        d = np.abs(c - r)
+    assert res["n_mismatch"] == np.count_nonzero(~close)
+    want_exact = 0
+    for i in range(n):
+        if c[i] == r[i]:
+            continue
+        if not (math.isfinite(c[i]) and math.isfinite(r[i])):
+            want_exact += 1
+            continue
+        di = abs(Fraction(c[i]) - Fraction(r[i]))
+        di = Fraction(float(di)) if di < Fraction(2) ** 1024 else None          # rounded once to binary64
+        t = Fraction(float(Fraction(rtol) * abs(Fraction(r[i]))))
+        tl = Fraction(float(Fraction(atol) + t))
+        want_exact += 0 if (di is not None and di <= tl) else 1
+    assert res["n_mismatch"] == want_exact
+    fin = np.isfinite(c) & np.isfinite(r)
+    assert res["n_nonfinite"] == np.count_nonzero(~fin) == 5 and res["flags"] == 1 | 2 | 4 | 8 | 16
+    assert res["max_abs"] == d[fin].max() == np.inf
+    nz = fin & (r != 0)
+    with np.errstate(all="ignore"):
+        assert res["max_rel"] == (d[nz] / np.abs(r[nz])).max()
+    assert res["sse"] == np.inf
+    # without the overflowing pair: the sum against math.fsum of exactly squared terms
+    c[special[6]] = r[special[6]] = 1.0
+    res = oracle.validate_f64(c, r, atol, rtol)
+    fin = np.isfinite(c) & np.isfinite(r)
+    dd = np.abs(c[fin] - r[fin])
+    want = float(sum(Fraction(float(x)) ** 2 for x in dd))
+    assert abs(res["sse"] - want) <= 1e-14 * want and res["max_abs"] == dd.max()
+    assert oracle.validate_f64(r[fin], r[fin], 0.0, 0.0)["pass"] == 1
+    assert oracle.validate_f64(np.zeros(0), np.zeros(0), 0.0, 0.0)["pass"] == 1
