@@ -61,8 +61,8 @@ enum {
 };
 
 /* Element types. EVO_U32 is accepted by evo_gen_inputs only; EVO_I32, EVO_I64 and EVO_U8 (also
- * the storage of bool) by evo_validate_exact only. */
-enum { EVO_U32 = 0, EVO_F32 = 1, EVO_F16 = 2, EVO_BF16 = 3, EVO_I32 = 5, EVO_I64 = 6, EVO_U8 = 7 };
+ * the storage of bool) by evo_validate_exact only; EVO_F64 by evo_validate_f64 only. */
+enum { EVO_U32 = 0, EVO_F32 = 1, EVO_F16 = 2, EVO_BF16 = 3, EVO_F64 = 4, EVO_I32 = 5, EVO_I64 = 6, EVO_U8 = 7 };
 
 /* Bits of evo_result.flags. */
 enum {
@@ -268,6 +268,26 @@ EVO_API int evo_validate_exact(evo_ctx* ctx, const void* const* cand_ptrs /* hos
                                const void* ref_ptr /* device */, const evo_desc* descs /* host */, uint64_t n_desc, int dtype,
                                evo_result_exact* results /* device */, uint32_t* group_pass /* device, optional */,
                                uint64_t n_group, void* stream);
+
+/*
+ * evo_validate_f64 - the correctness constraint for binary64 outputs.
+ * Paper: Section 3.1 Eq. 1 and Section 4.3, as evo_validate.  The same rule and statistics
+ * with every operation an individually rounded binary64 operation (no fused multiply-add on
+ * the rule's chain): d = |c - r|, tol = atol + rtol * |r|, close = (c == r) or (d finite and
+ * d <= tol); NaN/Inf elements are counted, flagged, judged by the rule and left out of
+ * max_abs, max_rel and sse.  Arguments as evo_validate; descriptor dtypes are EVO_F64 (or -1);
+ * tensors are aligned to 8 bytes (16-byte aligned ones take the vector path).
+ * Errors: EVO_ERR_ARG, EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_WORKSPACE, EVO_ERR_CUDA.
+ */
+typedef struct {
+    uint64_t n_mismatch, n_nonfinite;
+    double sse, max_abs, max_rel;
+    uint32_t flags, pass;
+} evo_result64;            /* 48 bytes */
+EVO_API int evo_validate_f64(evo_ctx* ctx, const void* const* cand_ptrs /* host array of device ptrs */,
+                             const void* ref_ptr /* device */, const evo_desc* descs /* host */, uint64_t n_desc,
+                             double atol, double rtol, evo_result64* results /* device */,
+                             uint32_t* group_pass /* device, optional */, uint64_t n_group, void* stream);
 
 /*
  * evo_mismatch_sample - where a failing candidate is wrong.

@@ -7,10 +7,10 @@ import numpy as np
 import torch
 
 EVO_U32, EVO_F32, EVO_F16, EVO_BF16 = 0, 1, 2, 3
-EVO_I32, EVO_I64, EVO_U8 = 5, 6, 7
+EVO_F64, EVO_I32, EVO_I64, EVO_U8 = 4, 5, 6, 7
 EVO_FLAG_INCOMPLETE = 0x40000000
 _TORCH_TO_CODE = {torch.float32: EVO_F32, torch.float16: EVO_F16, torch.bfloat16: EVO_BF16,
-                  torch.int32: EVO_I32, torch.int64: EVO_I64, torch.uint8: EVO_U8, torch.bool: EVO_U8}
+                  torch.float64: EVO_F64, torch.int32: EVO_I32, torch.int64: EVO_I64, torch.uint8: EVO_U8, torch.bool: EVO_U8}
 
 RESULT_DTYPE = np.dtype(
     [("n_mismatch", "<u8"), ("n_nonfinite", "<u8"), ("sse", "<f8"), ("max_abs", "<f4"),
@@ -25,6 +25,10 @@ EVO_STAT_MEDIAN, EVO_STAT_MEAN, EVO_STAT_MIN, EVO_STAT_TRIMMED_MEAN = 0, 1, 2, 3
 assert RESULT_DTYPE.itemsize == 40 and FIT_DTYPE.itemsize == 16 and _DESC_DTYPE.itemsize == 24
 EXACT_DTYPE = np.dtype([("n_mismatch", "<u8"), ("max_abs_diff", "<u8"), ("pass", "<u4"), ("pad", "<u4")], align=True)
 assert EXACT_DTYPE.itemsize == 24
+RESULT64_DTYPE = np.dtype(
+    [("n_mismatch", "<u8"), ("n_nonfinite", "<u8"), ("sse", "<f8"), ("max_abs", "<f8"), ("max_rel", "<f8"),
+     ("flags", "<u4"), ("pass", "<u4")], align=True)
+assert RESULT64_DTYPE.itemsize == 48
 OFFENDER_DTYPE = np.dtype([("index", "<u8"), ("cand", "<f4"), ("ref", "<f4")], align=True)
 assert SUMMARY_DTYPE.itemsize == 48 and OFFENDER_DTYPE.itemsize == 16
 
@@ -87,6 +91,8 @@ def load_library():
     L.evo_mismatch_sample.restype = i32
     L.evo_validate_exact.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp, u64, vp]
     L.evo_validate_exact.restype = i32
+    L.evo_validate_f64.argtypes = [vp, vp, vp, vp, u64, C.c_double, C.c_double, vp, vp, u64, vp]
+    L.evo_validate_f64.restype = i32
     _lib = L
     return L
 
@@ -239,6 +245,27 @@ def evo_validate_exact(cands, refs, groups=None, n_group=0, stream=None, ctx=Non
         _stream_ptr(stream, device))
     ctx.check(st)
     return results, group_pass
+
+
+def evo_validate_f64(cands, refs, atol, rtol, groups=None, n_group=0, stream=None, ctx=None):
+    """float64 CUDA tensors judged by the rule in binary64.  Returns (results: uint8 CUDA tensor of
+    len(cands) x 48 bytes, see results64_to_numpy; group_pass or None)."""
+    n = len(cands)
+    device = cands[0].device if n else torch.device("cuda", torch.cuda.current_device())
+    ctx = ctx or default_context(device.index)
+    ptrs, descs = _marshal(cands, refs, groups, is_host=False)
+    results = torch.empty((n, RESULT64_DTYPE.itemsize), dtype=torch.uint8, device=device)
+    group_pass = torch.empty(int(n_group), dtype=torch.int32, device=device) if groups is not None else None
+    st = load_library().evo_validate_f64(
+        ctx._h, C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(descs.ctypes.data), n, float(atol), float(rtol),
+        _dev_ptr(results), _dev_ptr(group_pass) if groups is not None else None,
+        int(n_group) if groups is not None else 0, _stream_ptr(stream, device))
+    ctx.check(st)
+    return results, group_pass
+
+
+def results64_to_numpy(results):
+    return results.cpu().numpy().view(RESULT64_DTYPE).reshape(-1)
 
 
 def exact_to_numpy(results):

@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libevo.so")
-SOURCES = ["context.cu", "plan.cu", "gen_inputs.cu", "validate.cu", "fitness.cu", "summary.cu", "feedback.cu", "validate_exact.cu"]
+SOURCES = ["context.cu", "plan.cu", "gen_inputs.cu", "validate.cu", "fitness.cu", "summary.cu", "feedback.cu", "validate_exact.cu", "validate_f64.cu"]
 
 NVCC_FLAGS = [
     "-std=c++17", "-O3", "-lineinfo",

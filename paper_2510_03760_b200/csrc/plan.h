@@ -60,7 +60,7 @@ inline uint32_t dtype_bytes(int dt) {
     switch (dt) {
         case EVO_F32: case EVO_I32: return 4;
         case EVO_F16: case EVO_BF16: return 2;
-        case EVO_I64: return 8;
+        case EVO_I64: case EVO_F64: return 8;
         case EVO_U8: return 1;
         default: return 0;
     }

@@ -27,7 +27,7 @@ def test_every_declared_function_is_exported(lib):
     assert {"evo_create", "evo_destroy", "evo_strerror", "evo_last_error", "evo_gen_inputs", "evo_validate",
             "evo_validate_host", "evo_fitness", "evo_fitness_host", "evo_plan_inspect", "evo_launch_count",
             "evo_set_timing_events", "evo_validate_static", "evo_validate_static_error", "evo_check",
-            "evo_selftest_wait", "evo_fitness_ex", "evo_summary", "evo_select_elite", "evo_mismatch_sample", "evo_validate_exact"} <= set(names)
+            "evo_selftest_wait", "evo_fitness_ex", "evo_summary", "evo_select_elite", "evo_mismatch_sample", "evo_validate_exact", "evo_validate_f64"} <= set(names)
     for n in names:
         assert hasattr(lib, n), n
 
