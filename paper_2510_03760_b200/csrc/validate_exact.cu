@@ -36,12 +36,15 @@ template <> struct IntElem<EVO_I32> {
     }
     static __device__ __forceinline__ void vec(const uint4& c, const uint4& r, uint32_t& cnt, unsigned long long& md) {
         const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, rw[4] = {r.x, r.y, r.z, r.w};
+        uint32_t m = 0;                                     // |c - r| of two int32 values fits 32 unsigned bits
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const unsigned long long d = diff(static_cast<int32_t>(cw[i]), static_cast<int32_t>(rw[i]));
+            const int32_t a = static_cast<int32_t>(cw[i]), b = static_cast<int32_t>(rw[i]);
+            const uint32_t d = a > b ? cw[i] - rw[i] : rw[i] - cw[i];
             cnt += d != 0 ? 1u : 0u;
-            md = d > md ? d : md;
+            m = max(m, d);
         }
+        md = m > md ? m : md;
     }
 };
 template <> struct IntElem<EVO_I64> {
@@ -154,6 +157,40 @@ __device__ __forceinline__ void run_set_exact(const SetRec& S, uint64_t t0, uint
     }
 }
 
+// A thread should keep about 128 bytes of every tensor in flight; a tile gives it 16 (uint8) or 64 (int32).
+// kGroup consecutive whole tiles are contiguous in memory, so they are taken together as one group with
+// kGroup times the vectors per thread; what does not fill a group goes through the generic routine tile by tile.
+// Functions of their own, so that their registers do not weigh on the other loops.
+template <int DT, int kGroup>
+__device__ __noinline__ void run_set_grouped(const SetRec& S, uint64_t t0, uint64_t t1, AccExact (*s_acc)[kWarps],
+                                             const void* const* s_cand, int warp, int lane) {
+    using E = IntElem<DT>;
+    constexpr int kTileVecs = kTileElems / E::kPerVec;
+    constexpr int kVecs = kGroup * kTileVecs / kThreads;                // vectors per thread per group
+    const uint64_t full_tiles = S.vec_ok ? S.n / kTileElems : 0;
+    uint64_t t = t0;
+    for (; t + kGroup <= t1 && t + kGroup <= full_tiles; t += kGroup) {
+        const uint64_t base = t * kTileVecs + threadIdx.x;
+        const uint4* rp = static_cast<const uint4*>(S.ref) + base;
+        uint4 r[kVecs];
+#pragma unroll
+        for (int v = 0; v < kVecs; ++v) r[v] = load_stream(rp + v * kThreads);
+#pragma unroll 1
+        for (uint32_t k = 0; k < S.k; ++k) {
+            const uint4* cp = static_cast<const uint4*>(s_cand[k]) + base;
+            uint4 c[kVecs];
+#pragma unroll
+            for (int v = 0; v < kVecs; ++v) c[v] = load_stream(cp + v * kThreads);
+            uint32_t cnt = 0;
+            unsigned long long md = 0;
+#pragma unroll
+            for (int v = 0; v < kVecs; ++v) E::vec(c[v], r[v], cnt, md);
+            commit(cnt, md, &s_acc[k][warp], lane);
+        }
+    }
+    if (t < t1) run_set_exact<DT>(S, t, t1, s_acc, s_cand, warp, lane);
+}
+
 __global__ void __launch_bounds__(kThreads, kCtasPerSmExact)
 exact_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members, const CtaRange* __restrict__ ranges,
             AccExact* __restrict__ partials) {
@@ -170,9 +207,9 @@ exact_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ membe
         for (uint32_t i = threadIdx.x; i < S.k * kWarps; i += kThreads) s_acc[i / kWarps][i % kWarps] = AccExact{0ull, 0ull};
         if (threadIdx.x < S.k) s_cand[threadIdx.x] = members[S.member_off + threadIdx.x].cand;
         __syncthreads();
-        if (S.dtype == EVO_I32) run_set_exact<EVO_I32>(S, t0, t1, s_acc, s_cand, warp, lane);
+        if (S.dtype == EVO_I32) run_set_grouped<EVO_I32, 2>(S, t0, t1, s_acc, s_cand, warp, lane);
         else if (S.dtype == EVO_I64) run_set_exact<EVO_I64>(S, t0, t1, s_acc, s_cand, warp, lane);
-        else run_set_exact<EVO_U8>(S, t0, t1, s_acc, s_cand, warp, lane);
+        else run_set_grouped<EVO_U8, 4>(S, t0, t1, s_acc, s_cand, warp, lane);
         __syncthreads();
         if (threadIdx.x < S.k) {
             AccExact a = s_acc[threadIdx.x][0];
