@@ -210,14 +210,34 @@ def _marshal(cands, refs, groups, is_host):
     return ptrs, descs
 
 
+class Prepared:
+    """The marshalled form of a population of CUDA tensors (pointer and descriptor arrays), built once
+    and reusable for any number of evo_validate calls on the same tensors: marshalling a few thousand
+    tensors in Python costs milliseconds, as much as checking them.  Keeps the tensors alive."""
+
+    def __init__(self, cands, refs, groups=None, n_group=0):
+        self.n = len(cands)
+        self.device = cands[0].device if self.n else torch.device("cuda", torch.cuda.current_device())
+        self.ptrs, self.descs = _marshal(cands, refs, groups, is_host=False)
+        self.has_groups = groups is not None
+        self.n_group = int(n_group) if self.has_groups else 0
+        self._keep = (list(cands), refs if isinstance(refs, torch.Tensor) else list(refs))
+
+
 def evo_validate(cands, refs, atol, rtol, groups=None, n_group=0, results=None, group_pass=None, stream=None, ctx=None):
     """Check CUDA tensors `cands[i]` against `refs[i]` (or one shared tensor).  Returns
     (results, group_pass): a uint8 CUDA tensor of len(cands) x 40 bytes (evo_result records,
-    see results_to_numpy) and, if `groups` is given, an int32 tensor of n_group verdicts."""
-    n = len(cands)
-    device = cands[0].device if n else torch.device("cuda", torch.cuda.current_device())
+    see results_to_numpy) and, if `groups` is given, an int32 tensor of n_group verdicts.
+    `cands` may be a Prepared population (then refs, groups and n_group are taken from it)."""
+    if isinstance(cands, Prepared):
+        prep = cands
+        n, device, ptrs, descs = prep.n, prep.device, prep.ptrs, prep.descs
+        groups, n_group = (True if prep.has_groups else None), prep.n_group
+    else:
+        n = len(cands)
+        device = cands[0].device if n else torch.device("cuda", torch.cuda.current_device())
+        ptrs, descs = _marshal(cands, refs, groups, is_host=False)
     ctx = ctx or default_context(device.index)
-    ptrs, descs = _marshal(cands, refs, groups, is_host=False)
     if results is None:
         results = torch.empty((n, RESULT_DTYPE.itemsize), dtype=torch.uint8, device=device)
     if groups is not None and group_pass is None:

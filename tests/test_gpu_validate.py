@@ -181,6 +181,22 @@ def test_results_are_reproducible_and_independent_of_other_tensors(evo):
     assert_results_equal(evo.results_to_numpy(res), a[7:8])
 
 
+def test_prepared_population_gives_the_same_results(evo):
+    pop = workloads.config5("cpu", n_cand=30, log2_min=8.0, log2_max=15.0, trials=4)
+    dev_refs = [r.cuda() for r in pop.refs]
+    cands = [t.cand.cuda() for t in pop.tensors]
+    refs = [dev_refs[t.ref_index] for t in pop.tensors]
+    groups = [t.group for t in pop.tensors]
+    res, gp = evo.evo_validate(cands, refs, pop.atol, pop.rtol, groups=groups, n_group=pop.n_group)
+    prep = evo.Prepared(cands, refs, groups, pop.n_group)
+    for _ in range(2):
+        res2, gp2 = evo.evo_validate(prep, None, pop.atol, pop.rtol)
+        assert torch.equal(res, res2) and torch.equal(gp, gp2)
+    prep_ng = evo.Prepared(cands, refs)
+    res3, gp3 = evo.evo_validate(prep_ng, None, pop.atol, pop.rtol)
+    assert torch.equal(res, res3) and gp3 is None
+
+
 def test_empty_call_and_empty_groups(evo):
     res, gp = evo.evo_validate([], [], 0.1, 0.1, groups=[], n_group=3)
     torch.cuda.synchronize()
