@@ -656,15 +656,24 @@ seed_kernel(const SetRec* __restrict__ sets, const MemberRec* __restrict__ membe
     __shared__ uint32_t s_max[kWarps];
     const MemberRec M = members[blockIdx.x];
     const SetRec S = sets[M.set];
-    const uint64_t n = S.n < static_cast<uint64_t>(kTileElems) ? S.n : static_cast<uint64_t>(kTileElems);
+    const uint32_t n = static_cast<uint32_t>(S.n < static_cast<uint64_t>(kTileElems) ? S.n : static_cast<uint64_t>(kTileElems));
+    // all 16 element pairs of the thread are loaded before any is used: one round of memory latency, not sixteen
+    float c[kEpt], r[kEpt];
+#pragma unroll
+    for (int j = 0; j < kEpt; ++j) {
+        const uint32_t e = threadIdx.x + j * kThreads;
+        c[j] = 0.f; r[j] = 0.f;
+        if (e < n) {
+            if (S.dtype == EVO_F32) { c[j] = static_cast<const float*>(M.cand)[e]; r[j] = static_cast<const float*>(S.ref)[e]; }
+            else if (S.dtype == EVO_F16) { c[j] = __half2float(static_cast<const __half*>(M.cand)[e]); r[j] = __half2float(static_cast<const __half*>(S.ref)[e]); }
+            else { c[j] = __bfloat162float(static_cast<const __nv_bfloat16*>(M.cand)[e]); r[j] = __bfloat162float(static_cast<const __nv_bfloat16*>(S.ref)[e]); }
+        }
+    }
     float best = 0.f;
-    for (uint64_t e = threadIdx.x; e < n; e += kThreads) {
-        float c, r;
-        if (S.dtype == EVO_F32) { c = static_cast<const float*>(M.cand)[e]; r = static_cast<const float*>(S.ref)[e]; }
-        else if (S.dtype == EVO_F16) { c = __half2float(static_cast<const __half*>(M.cand)[e]); r = __half2float(static_cast<const __half*>(S.ref)[e]); }
-        else { c = __bfloat162float(static_cast<const __nv_bfloat16*>(M.cand)[e]); r = __bfloat162float(static_cast<const __nv_bfloat16*>(S.ref)[e]); }
-        const float d = fabsf(__fsub_rn(c, r)), ar = fabsf(r);
-        const bool usable = d > 0.f && ar > 0.f && d < kInf && ar < kInf && fabsf(c) < kInf;      // as the statistics: finite pairs, r != 0
+#pragma unroll
+    for (int j = 0; j < kEpt; ++j) {
+        const float d = fabsf(__fsub_rn(c[j], r[j])), ar = fabsf(r[j]);
+        const bool usable = d > 0.f && ar > 0.f && d < kInf && ar < kInf && fabsf(c[j]) < kInf;   // as the statistics: finite pairs, r != 0
         if (usable) best = fmaxf(best, __fdiv_rn(d, ar));
     }
     const uint32_t w = __reduce_max_sync(0xffffffffu, __float_as_uint(best));
