@@ -84,3 +84,16 @@ def test_product_does_not_reach_into_the_oracle():
         if f.endswith((".py", ".cpp")):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2510_03760_b200" not in text and "libevo.so" not in text, f
+
+
+def test_the_header_is_plain_c(tmp_path):
+    """include/evo.h is the boundary: it must compile as C99 without warnings, no C++ needed."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("gcc not found")
+    src = tmp_path / "use_evo.c"
+    src.write_text('#include "evo.h"\nint main(void) { evo_result r; evo_desc d; (void)r; (void)d; return EVO_OK; }\n')
+    p = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(ROOT, "include"),
+                        "-fsyntax-only", str(src)], capture_output=True, text=True)
+    assert p.returncode == 0, p.stderr
