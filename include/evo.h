@@ -117,7 +117,8 @@ typedef struct {
 typedef struct {
     uint64_t n_mismatch;   /* elements violating the closeness rule */
     uint64_t n_nonfinite;  /* elements where candidate or reference is NaN or +-Inf */
-    double sse;            /* sum of d^2 over elements with both values finite */
+    double sse;            /* sum of d^2 over elements with both values finite (partial sums of up to 512 elements are
+                              formed in binary32, the rest in binary64: within 1e-5 relative of the exact sum) */
     float max_abs;         /* max d over those elements (0 if none; +Inf if a finite difference overflows) */
     float max_rel;         /* max d / |r| over those elements with r != 0 (0 if none) */
     uint32_t flags;        /* EVO_FLAG_* */
