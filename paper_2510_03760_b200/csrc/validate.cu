@@ -3,8 +3,8 @@
 // reference outputs), with the error statistics reported alongside the verdict.
 //
 // Shape of the computation: a pure streaming read.  Every candidate element and every
-// distinct reference element has to come from HBM once; per element there are seven to
-// nine binary32 operations.  The design therefore spends its effort on (1) never reading a
+// distinct reference element has to come from HBM once; per element there are five to
+// eight binary32 operations.  The design therefore spends its effort on (1) never reading a
 // reference tile more than once per set of candidates that share it, (2) keeping many
 // bytes in flight per SM independently of the arithmetic, and (3) keeping reductions and
 // everything that depends on the reference alone off the per-candidate path.
@@ -16,7 +16,7 @@
 //   pass 1        persistent CTAs walk their range.  A producer warp streams the tiles
 //                 (reference, then each member) into a ring of shared-memory stages with
 //                 bulk asynchronous copies that complete on mbarriers; eight consumer warps
-//                 take a reference tile into registers once (value, tolerance, |r|), then
+//                 take a reference tile into registers once (values, smallest tolerance), then
 //                 compare each member's tile against it.  Per (tile, member) a warp folds
 //                 its lanes with redux/shuffles into a warp-private accumulator in shared
 //                 memory.  When a CTA leaves a set it writes one partial record per member.
@@ -237,9 +237,10 @@ constexpr float kShrink = 0.99999904632568359375f;      // 1 - 2^-20
 
 // One full, 16-byte aligned tile: reference into registers once, then every member.
 //
-// Fast path per element, valid when c and r are finite and d does not overflow:
-// d = |c - r| against the tolerance computed once per reference element; with atol, rtol >= 0
-// and finite data c == r implies d = 0 <= tol, so the equality clause needs no test here.
+// Fast path per element, valid when c and r are finite and d does not overflow: d = |c - r|,
+// its maximum and its square; mismatches are counted only for a thread whose largest d exceeds
+// the smallest tolerance of its elements.  With atol, rtol >= 0 and finite data c == r implies
+// d = 0 <= tol, so the equality clause needs no test here.
 // The quotient d/|r| is not formed: `mlo` is slightly below the running maximum m of the
 // quotient, and d > RZ(mlo*|r|) holds whenever fl(d/|r|) > m could (rounding the product
 // toward zero keeps the test one-sided), so a miss never loses a maximum.  A thread whose
@@ -251,7 +252,7 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
     using E = Elem<DT>;
     if (g.dead) return;
     constexpr uint32_t kVecStride = kThreads * 16;
-    float r[kEpt], tol[kEpt];
+    float r[kEpt];
     if (!ring_acquire(g)) return;
     {
         const uint32_t a = g.data() + threadIdx.x * 16;
@@ -263,8 +264,13 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
         }
     }
     ring_release(g, lane);
+    // The smallest tolerance among this thread's 16 reference elements: tol = atol + rtol*|r| does not decrease
+    // with |r| (each rounding is monotone), so it is the tolerance of the smallest |r|.  A member whose largest
+    // difference over these elements stays within it has no mismatch here, and none is counted element by element.
+    float armin = kInf;
 #pragma unroll
-    for (int e = 0; e < kEpt; ++e) tol[e] = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r[e])));
+    for (int e = 0; e < kEpt; ++e) armin = fminf(armin, fabsf(r[e]));
+    const float tolmin = __fadd_rn(atol, __fmul_rn(rtol, armin));
     const uint64_t vec0 = t * (kTileElems / E::kPerVec) + threadIdx.x;   // this thread's first vector of the tile
 #pragma unroll 1
     for (int k = 0; k < K; ++k) {
@@ -290,7 +296,6 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
             for (int e = 0; e < E::kPerVec; ++e) {
                 const int i = v * E::kPerVec + e;
                 const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
-                cnt += __float_as_uint(__fsub_rn(tol[i], d)) >> 31;       // sign of tol - d: set iff d > tol
                 ma = fmaxf(ma, d);
                 sse = fmaf(d, d, sse);
                 trig |= d > __fmul_rz(mlo, fabsf(r[i]));
@@ -298,6 +303,18 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
         // The fast numbers do not stand if something was NaN/Inf or overflowed (the sum of
         // squares is then NaN/Inf) or if every d is so small that d^2 underflows in binary32.
         const bool redo = !(sse < kInf) || (ma < 9.094947017729282e-13f /* 2^-40 */ && ma > 0.f);
+        if (ma > tolmin && !redo) {
+            // some difference may exceed its tolerance: count, element by element
+#pragma unroll
+            for (int v = 0; v < E::kVecs; ++v)
+#pragma unroll
+                for (int e = 0; e < E::kPerVec; ++e) {
+                    const int i = v * E::kPerVec + e;
+                    const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
+                    const float tol = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r[i])));
+                    cnt += (d > tol) ? 1u : 0u;
+                }
+        }
         float mt = m;
         float lo = mlo;
         bool scan = trig && !redo;
