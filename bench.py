@@ -355,6 +355,11 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    # how evenly the fixed cut spreads the tiles over the persistent CTAs (host-side view of the schedule)
+    pi = evo.plan_inspect(cands, refs, 2 * torch.cuda.get_device_properties(device).multi_processor_count)
+    w = pi["weights"]
+    plan_info = {"n_sets": pi["n_sets"], "n_ctas": pi["n_ctas"], "total_tiles": pi["total_tiles"],
+                 "max_over_mean_tiles_per_cta": float(w.max() / w.mean()) if len(w) else None}
     peak, peak_kind = measured_peak()
     kern_avg_ms = sum(kern_ms) / len(kern_ms)
     achieved = alg_bytes / (kern_avg_ms * 1e-3) / 1e9
@@ -381,6 +386,7 @@ def run_ours(args):
                    "algorithmic_bytes_per_step": alg_bytes, "l2": "inputs larger than L2" if alg_bytes > (1 << 28) else "inputs fit in L2",
                    "replicas": world},
         "candidates_per_s": cand_per_s, "frac_of_hbm_peak": value / world / peak,
+        "candidate_bytes_gbs": world * pop.candidate_bytes() / (ms_per_step * 1e-3) / 1e9, "plan": plan_info,
         "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "cpu_baseline": cpu,
     }

@@ -93,6 +93,8 @@ def load_library():
     L.evo_validate_exact.restype = i32
     L.evo_validate_f64.argtypes = [vp, vp, vp, vp, u64, C.c_double, C.c_double, vp, vp, u64, vp]
     L.evo_validate_f64.restype = i32
+    L.evo_plan_inspect.argtypes = [vp, vp, vp, u64, i32, u32, vp, vp, vp, vp]
+    L.evo_plan_inspect.restype = i32
     _lib = L
     return L
 
@@ -248,6 +250,41 @@ def evo_validate(cands, refs, atol, rtol, groups=None, n_group=0, results=None, 
         int(n_group) if groups is not None else 0, _stream_ptr(stream, device))
     ctx.check(st)
     return results, group_pass
+
+
+_PLAN_SUMMARY = np.dtype([("n_sets", "<u4"), ("n_ctas", "<u4"), ("n_parts", "<u4"), ("tile_elems", "<u4"),
+                          ("total_tiles", "<u8")], align=True)
+_PLAN_RANGE = np.dtype([("tile_begin", "<u8"), ("tile_end", "<u8"), ("set_begin", "<u4"), ("set_end", "<u4")], align=True)
+
+
+def plan_inspect(cands, refs, max_ctas):
+    """The schedule evo_validate would use for these CUDA tensors on a device running `max_ctas` persistent CTAs
+    (evo_plan_inspect; host only).  Returns a dict: n_sets, n_ctas, total_tiles, tile_elems, and `weights`, the
+    tiles each CTA moves (tiles of its run times members + 1), as a numpy array."""
+    ptrs, descs = _marshal(cands, refs, None, is_host=False)
+    n = len(cands)
+    summ = np.zeros(1, _PLAN_SUMMARY)
+    ranges = np.zeros(int(max_ctas), _PLAN_RANGE)
+    set_of = np.zeros(max(n, 1), np.uint32)
+    set_k = np.zeros(max(n, 1), np.uint32)
+    st = load_library().evo_plan_inspect(C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(descs.ctypes.data), n, EVO_F32,
+                                         int(max_ctas), C.c_void_p(summ.ctypes.data), C.c_void_p(ranges.ctypes.data),
+                                         C.c_void_p(set_of.ctypes.data), C.c_void_p(set_k.ctypes.data))
+    if st != 0:
+        raise EvoError(st, load_library().evo_strerror(st).decode())
+    s = summ[0]
+    te = int(s["tile_elems"])
+    set_tiles = np.zeros(int(s["n_sets"]), np.int64)
+    for i in range(n):
+        set_tiles[set_of[i]] = (int(descs["n"][i]) + te - 1) // te
+    weights = np.zeros(int(s["n_ctas"]), np.int64)
+    for b, r in enumerate(ranges[: int(s["n_ctas"])]):
+        for q in range(int(r["set_begin"]), int(r["set_end"]) + 1):
+            t0 = int(r["tile_begin"]) if q == r["set_begin"] else 0
+            t1 = int(r["tile_end"]) if q == r["set_end"] else int(set_tiles[q])
+            weights[b] += max(0, t1 - t0) * (int(set_k[q]) + 1)
+    return {"n_sets": int(s["n_sets"]), "n_ctas": int(s["n_ctas"]), "total_tiles": int(s["total_tiles"]),
+            "tile_elems": te, "weights": weights}
 
 
 def evo_validate_exact(cands, refs, groups=None, n_group=0, stream=None, ctx=None):

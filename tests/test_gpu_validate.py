@@ -197,6 +197,14 @@ def test_prepared_population_gives_the_same_results(evo):
     assert torch.equal(res, res3) and gp3 is None
 
 
+def test_plan_inspect_through_the_binding(evo):
+    ref = torch.zeros(1 << 22, device="cuda")
+    cands = [torch.zeros(1 << 22, device="cuda") for _ in range(16)]
+    info = evo.plan_inspect(cands, [ref] * 16, 296)
+    assert info["n_sets"] == 1 and info["n_ctas"] == 296 and info["total_tiles"] == 1024 and info["tile_elems"] == 4096
+    assert info["weights"].sum() == 1024 * 17 and info["weights"].max() <= 4 * 17
+
+
 def test_empty_call_and_empty_groups(evo):
     res, gp = evo.evo_validate([], [], 0.1, 0.1, groups=[], n_group=3)
     torch.cuda.synchronize()
