@@ -18,16 +18,30 @@ constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
 constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
 constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
 
-__device__ __forceinline__ uint4 philox4x32_10(uint64_t block, uint32_t k0, uint32_t k1) {
+// The ten round keys (key bumped by the Weyl constants before every round but the first) depend on the seed
+// only: the host works them out once and passes them as a kernel argument, so a round reads them as constant
+// operands instead of spending two additions.
+struct RoundKeys { uint32_t k0[10], k1[10]; };
+
+inline RoundKeys round_keys(uint64_t seed) {
+    RoundKeys rk;
+    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
+    for (int round = 0; round < 10; ++round) {
+        rk.k0[round] = k0; rk.k1[round] = k1;
+        k0 += kPhiloxW0; k1 += kPhiloxW1;
+    }
+    return rk;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint64_t block, const RoundKeys& rk) {
     uint32_t c0 = static_cast<uint32_t>(block), c1 = static_cast<uint32_t>(block >> 32), c2 = 0u, c3 = 0u;
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
         const uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
         const uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
-        const uint32_t n0 = hi1 ^ c1 ^ k0;
-        const uint32_t n2 = hi0 ^ c3 ^ k1;
+        const uint32_t n0 = hi1 ^ c1 ^ rk.k0[round];
+        const uint32_t n2 = hi0 ^ c3 ^ rk.k1[round];
         c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-        k0 += kPhiloxW0; k1 += kPhiloxW1;
     }
     return make_uint4(c0, c1, c2, c3);
 }
@@ -56,13 +70,12 @@ template <int DT> struct alignas(4 * sizeof(typename Out<DT>::T)) Quad { typenam
 // [offset, offset + n); `lead` = offset mod 4 elements of the first block are skipped.
 // VEC: lead == 0 and `out` is aligned for one store of four elements per block.
 template <int DT, bool VEC>
-__global__ void __launch_bounds__(256) gen_kernel(uint64_t seed, uint64_t first_block, uint64_t n_blocks,
+__global__ void __launch_bounds__(256) gen_kernel(const __grid_constant__ RoundKeys rk, uint64_t first_block, uint64_t n_blocks,
                                                   uint32_t lead, uint64_t n, typename Out<DT>::T* __restrict__ out) {
     using T = typename Out<DT>::T;
-    const uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     for (uint64_t j = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n_blocks; j += stride) {
-        const uint4 w = philox4x32_10(first_block + j, k0, k1);
+        const uint4 w = philox4x32_10(first_block + j, rk);
         Quad<DT> q;
         if (DT == EVO_U32) {
             q.v[0] = Out<DT>::make(w.x, 0.f); q.v[1] = Out<DT>::make(w.y, 0.f);
@@ -93,8 +106,9 @@ cudaError_t launch(evo_ctx* ctx, uint64_t seed, uint64_t offset, uint64_t n, voi
     const uint64_t want = (n_blocks + 255) / 256;
     const uint64_t cap = static_cast<uint64_t>(ctx->sm_count) * 8 * 4;   // a few waves of 8 resident CTAs per SM
     const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
-    if (vec) gen_kernel<DT, true><<<grid, 256, 0, stream>>>(seed, offset >> 2, n_blocks, lead, n, static_cast<T*>(out));
-    else     gen_kernel<DT, false><<<grid, 256, 0, stream>>>(seed, offset >> 2, n_blocks, lead, n, static_cast<T*>(out));
+    const RoundKeys rk = round_keys(seed);
+    if (vec) gen_kernel<DT, true><<<grid, 256, 0, stream>>>(rk, offset >> 2, n_blocks, lead, n, static_cast<T*>(out));
+    else     gen_kernel<DT, false><<<grid, 256, 0, stream>>>(rk, offset >> 2, n_blocks, lead, n, static_cast<T*>(out));
     ctx->launches += 1;
     return cudaGetLastError();
 }
