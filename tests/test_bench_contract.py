@@ -30,3 +30,26 @@ def test_ranks_other_than_zero_of_the_reference_arm_do_no_work():
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "2"],
                        capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
     assert p.returncode == 0 and p.stdout.strip() == ""
+
+
+import pytest
+
+
+@pytest.mark.gpu
+def test_gpu_arm_prints_one_json_line_with_roofline_e2e_and_cpu_baseline():
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "config2", "--steps", "20", "--warmup", "3"],
+                       capture_output=True, text=True, timeout=900, cwd=ROOT)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [l for l in p.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    j = json.loads(lines[0])
+    assert j["metric"] == "validated_bytes_per_second" and j["unit"] == "GB/s" and j["n_gpus"] == 1 and j["steps"] == 20
+    assert j["value"] > 0 and j["scaling"] == "weak" and j["dtype"] == "f32" and j["config"]["workload"] == "config2"
+    assert j["gpu_launches"] >= 6 * 20                      # gen, pass 1, pass 2, verdicts, two fitness launches per step
+    r = j["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 0 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    e = j["e2e"]
+    assert e["value"] > 0 and e["h2d_bytes_per_step"] >= j["config"]["algorithmic_bytes_per_step"] and e["d2h_bytes_per_step"] > 0
+    c = j["cpu_baseline"]
+    assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["sample"]
+    assert set(j["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
