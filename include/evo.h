@@ -276,7 +276,9 @@ EVO_API int evo_validate_exact(evo_ctx* ctx, const void* const* cand_ptrs /* hos
  * with every operation an individually rounded binary64 operation (no fused multiply-add on
  * the rule's chain): d = |c - r|, tol = atol + rtol * |r|, close = (c == r) or (d finite and
  * d <= tol); NaN/Inf elements are counted, flagged, judged by the rule and left out of
- * max_abs, max_rel and sse (sse is summed in binary64: squares below its range are lost).
+ * max_abs, max_rel and sse (every square d*d is a binary64 product, so a square below the
+ * binary64 range is lost and one in its subnormal range keeps only the bits that fit; the sum of
+ * the squares is within 1e-12 relative of their exact sum).
  * Arguments as evo_validate; descriptor dtypes are EVO_F64 (or -1);
  * tensors are aligned to 8 bytes (16-byte aligned ones take the vector path).
  * Errors: EVO_ERR_ARG, EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_WORKSPACE, EVO_ERR_CUDA.

@@ -582,8 +582,11 @@ extern "C" void oracle_group_pass_exact(const oracle_result_exact* results, cons
 // operation an individually rounded binary64 operation (no fused multiply-add):
 // d = |c - r|, tol = atol + rtol*|r|, close = (c == r) or (d finite and d <= tol);
 // NaN/Inf elements are counted and flagged and stay out of max_abs, max_rel and
-// sse.  The sum of squares is accumulated in extended precision (long double) so
-// that the oracle's own summation error stays far below the comparison bar.
+// sse.  The square is one more individually rounded binary64 operation (a square
+// below the binary64 range is lost, one in its subnormal range keeps only the bits
+// that fit); the rounded squares are then accumulated in extended precision (long
+// double) so that the oracle's own summation error stays far below the comparison
+// bar.
 // ---------------------------------------------------------------------------
 struct oracle_result64 {
     uint64_t n_mismatch, n_nonfinite;
@@ -610,7 +613,8 @@ extern "C" int oracle_validate_f64(const double* cand, const double* ref, uint64
         if (f) { ++res.n_nonfinite; res.flags |= f; continue; }
         if (d > res.max_abs) res.max_abs = d;
         if (r != 0.0) { const double q = d / std::fabs(r); if (q > res.max_rel) res.max_rel = q; }
-        sse += static_cast<long double>(d) * static_cast<long double>(d);
+        const double sq = d * d;                      // rounded once to binary64
+        sse += static_cast<long double>(sq);
     }
     res.sse = static_cast<double>(sse);
     res.pass = res.n_mismatch == 0 ? 1u : 0u;

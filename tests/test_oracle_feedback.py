@@ -146,3 +146,38 @@ def test_binary64_rule_against_numpy_isclose_exact_rationals_and_fsum():
     assert abs(res["sse"] - want) <= 1e-14 * want and res["max_abs"] == dd.max()
     assert oracle.validate_f64(r[fin], r[fin], 0.0, 0.0)["pass"] == 1
     assert oracle.validate_f64(np.zeros(0), np.zeros(0), 0.0, 0.0)["pass"] == 1
+
+
+def test_binary64_squares_are_rounded_to_binary64_before_they_are_summed():
+    """The sum of squares of the binary64 rule sums d*d as binary64 products: a square below the binary64
+    range counts as 0, one in the subnormal range keeps only the bits that fit.  Checked with exact rationals."""
+    from fractions import Fraction
+    rng = np.random.default_rng(31)
+    n = 4000
+    r = rng.standard_normal(n)
+
+    def defined_and_exact(c, r):
+        d = [abs(Fraction(float(a)) - Fraction(float(b))) for a, b in zip(c, r)]
+        d = [Fraction(float(x)) for x in d]                       # the difference, rounded once
+        exact = sum(x * x for x in d)
+        defined = sum(Fraction(float(x * x)) for x in d)          # each square rounded once, then summed exactly
+        return float(defined), exact
+
+    # (a) every square is below the smallest subnormal: the exact sum is positive, the defined one is 0
+    ra = r * 1e-170
+    ca = ra * (1 + 2.0 ** -20)
+    defined, exact = defined_and_exact(ca, ra)
+    assert exact > 0 and defined == 0.0
+    assert oracle.validate_f64(ca, ra, 0.0, 0.0)["sse"] == 0.0
+    # (b) squares in the subnormal range: sums of multiples of 2^-1074 are exact, so the value is fixed bit for bit
+    rb = r * 1e-155
+    cb = rb * (1 + 2.0 ** -10)
+    defined, exact = defined_and_exact(cb, rb)
+    assert 0 < defined < 2.0 ** -1022 and Fraction(defined) != exact
+    assert oracle.validate_f64(cb, rb, 0.0, 0.0)["sse"] == defined
+    # (c) normal squares with lost ones among them: the defined sum within the summation's own error
+    rc = np.where(np.arange(n) % 2 == 0, r, r * 1e-170)
+    cc = rc * (1 + 2.0 ** -20)
+    defined, exact = defined_and_exact(cc, rc)
+    got = oracle.validate_f64(cc, rc, 0.0, 0.0)["sse"]
+    assert abs(got - defined) <= 1e-15 * defined
