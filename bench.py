@@ -8,11 +8,15 @@ rate at which candidate outputs are validated: algorithmic bytes (every candidat
 every distinct reference once) per second, for inputs already resident in HBM (`value`) and
 through the host-buffer entry points with the copies inside the timed region (`e2e`).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4|config3|config5|config2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4|config3|config5|config2|config1]
     python bench.py --impl reference ...     # the CPU oracle on a bounded sample (baseline arm)
 
-With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank evaluates its own
-replica of the population: candidates are independent, there is no exchange between GPUs.
+With N > 1 every rank evaluates its own replica of the population (one rank per GPU): candidates
+are independent, there is no exchange between GPUs.  Started without a launcher, `--gpus N`
+re-executes itself under torch.distributed.run with N local ranks.
+
+The default run (config 4) also reports, under "per_config", the other synthetic populations
+(configs 1, 2, 3 and 5): time of the main kernel, of the evo_validate call and of the whole step.
 """
 import argparse
 import json
@@ -32,7 +36,9 @@ import workloads  # noqa: E402
 
 METRIC = "validated_bytes_per_second"
 UNIT = "GB/s"
+DATASHEET_HBM_GBS = 7700.0      # nominal HBM3e bandwidth of a 180 GB B200 (HGX figure; the DGX figure is 8000)
 WORKLOAD_NOTES = {
+    "config1": "1 fp32 candidate of 64 x 64 elements against its reference (fits in L2; latency)",
     "config4": "16 fp32 candidates x 2^28 elements (1 GiB each) sharing one 1 GiB reference",
     "config3": "64 fp16 + 64 bf16 candidates x 2^20 elements, one reference per dtype",
     "config5": "1024 candidates, 1-3 tensors each, 2^10..2^24 elements, fp32/fp16/bf16, own references",
@@ -61,8 +67,8 @@ def measured_peak():
 
 
 # DRAM traffic of validate_pass1 as counted by ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a reduced
-# config 4 (2^24 elements per tensor), per algorithmic byte; see profiles/validate_pass1_config4_2p24.md.
-# It stands only for the kernel sources it was captured on: their hash is checked.
+# config 4 (2^24 elements per tensor), per algorithmic byte (the capture is summarised under profiles/).
+# It stands only for the kernel sources it was captured on: their hash is checked, and a mismatch reports null.
 NCU_TRAFFIC = {"dram_bytes_per_algorithmic_byte": 1.006, "sources_sha1": "bb401ccbd21d8636dbe08b0724bdf0740fec5a78"}
 
 
@@ -141,21 +147,25 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- oracle arm
-FULL_SHAPE = {"config4": dict(n=1 << 28, k=16), "config3": dict(n=1 << 20, k=128), "config2": dict(n=1 << 18, k=8)}
+FULL_SHAPE = {"config4": dict(n=1 << 28, k=16), "config3": dict(n=1 << 20, k=128), "config2": dict(n=1 << 18, k=8),
+              "config1": dict(n=1 << 12, k=1)}
+FULL_TRIALS = {"config1": 5}
 
 
 class OracleSample:
     """A bounded sample of a workload for the CPU oracle, and the factors that scale its
     timings (linear in elements) to one full step of that workload."""
 
-    def __init__(self, workload, log2_elems, log2_gen):
+    def __init__(self, workload, log2_elems, log2_gen, seed=None):
         if workload in FULL_SHAPE:
             n_full, k_full = FULL_SHAPE[workload]["n"], FULL_SHAPE[workload]["k"]
             n_s = min(n_full, 1 << log2_elems)
             if workload == "config4":
-                pop = workloads.config4("cpu", n=n_s, k=4)
+                pop = workloads.config4("cpu", n=n_s, k=4, **({} if seed is None else {"seed": seed}))
             elif workload == "config3":
                 pop = workloads.config3("cpu", n=n_s, k_per_dtype=2)
+            elif workload == "config1":
+                pop = workloads.config1("cpu")
             else:
                 pop = workloads.config2("cpu", n=n_s, k=4)
             self.scale_val = (n_full * k_full) / float(n_s * len(pop.tensors))
@@ -173,8 +183,8 @@ class OracleSample:
         import numpy as np
         self.times = np.repeat(pop.times.numpy()[:1], self.rows, axis=0)
         self.base = pop.base_times.numpy()
-        self.description = ("oracle, 1 thread: validate %s, generate 2^%d normals, fitness of %d rows; "
-                            "timings scaled linearly in elements to one full step" % (what, self.n_gen.bit_length() - 1, self.rows))
+        self.what = "validate %s, generate 2^%d normals, fitness of %d rows" % (what, self.n_gen.bit_length() - 1, self.rows)
+        self.description = ("oracle, 1 thread: %s; timings scaled linearly in elements to one full step" % self.what)
 
     def run(self):
         """One timed pass over the sample; returns (estimated seconds of a full step, seconds spent)."""
@@ -191,18 +201,71 @@ class OracleSample:
         return est, t3 - t0
 
 
+# The sample both oracle legs time (the reference arm once per step, the cpu_baseline leg a few times over):
+# log2 of the elements per sampled tensor and of the generated normals.
+ORACLE_SAMPLE_LOG2 = (24, 22)
+
+
 def full_algorithmic_bytes(workload):
-    known = {"config4": 17 * (1 << 30), "config3": 130 * (1 << 21), "config2": 9 * (1 << 20)}
+    known = {"config4": 17 * (1 << 30), "config3": 130 * (1 << 21), "config2": 9 * (1 << 20), "config1": 2 * (1 << 14)}
     return known.get(workload, int(2048 * 1.73e6 * 3 * 2))
 
 
+def config_keys(workload, n_gen, n_tensors, n_group, trials, alg_bytes, world):
+    """The `config` object of a line: the same keys, built the same way, in both arms."""
+    return {"workload": workload, "what": WORKLOAD_NOTES[workload],
+            "step": "evo_gen_inputs(%d fp32 normals) + evo_validate(%d tensors) + evo_fitness(%d x %d trials)"
+                    % (n_gen, n_tensors, n_group, trials),
+            "algorithmic_bytes_per_step": alg_bytes,
+            "l2": "inputs larger than L2" if alg_bytes > (1 << 28) else "inputs fit in L2", "replicas": world}
+
+
+def _oracle_process(workload, seed, passes, barrier, queue):
+    """One worker of the many-process baseline: its own sample (other tensors than every other worker's),
+    built before the common start, then `passes` timed passes."""
+    sample = OracleSample(workload, ORACLE_SAMPLE_LOG2[0], ORACLE_SAMPLE_LOG2[1], seed=seed)
+    sample.run()
+    barrier.wait()
+    t0 = time.perf_counter()
+    ests = [sample.run()[0] for _ in range(passes)]
+    queue.put((sum(ests) / len(ests), time.perf_counter() - t0, sample.what))
+
+
+def oracle_many_processes(workload, alg_bytes, passes):
+    """The oracle as P independent single-threaded processes over disjoint candidates, P = the cores this process may
+    use.  Processes are spawned (never forked: the parent holds a CUDA context).  Returns the cpu_baseline-style dict."""
+    import multiprocessing as mp
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    ctx = mp.get_context("spawn")
+    barrier, queue = ctx.Barrier(cores + 1), ctx.Queue()
+    procs = [ctx.Process(target=_oracle_process, args=(workload, 4000 + 17 * (i + 1), passes, barrier, queue), daemon=True)
+             for i in range(cores)]
+    for p in procs:
+        p.start()
+    try:
+        barrier.wait(timeout=600)
+        t0 = time.perf_counter()
+        got = [queue.get(timeout=600) for _ in procs]
+        wall = time.perf_counter() - t0
+    finally:
+        for p in procs:
+            p.join(timeout=30)
+            if p.is_alive():
+                p.kill()
+    rate = sum(alg_bytes / g[0] for g in got) / 1e9
+    return {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle, one single-threaded process per core, disjoint candidates",
+            "sample": "each process: %d passes over its own sample (%s); the rates of the processes added up" % (passes, got[0][2]),
+            "seconds": wall}
+
+
 def run_reference(args):
-    """Baseline arm: the CPU oracle, as it stands, on the host cores; rank 0 only."""
+    """Baseline arm: the CPU oracle, as it stands, on the host cores; rank 0 only.  Every step is one pass over a
+    bounded sample of the workload; `value` scales the sample's timings to a full step."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     passes = args.steps + args.warmup
-    log2 = 24 if passes <= 30 else 22 if passes <= 120 else 20 if passes <= 500 else 18   # about 1 s .. 20 ms per pass
-    sample = OracleSample(args.workload, log2, log2 - 2)
+    shrink = 0 if passes <= 30 else 2 if passes <= 120 else 4 if passes <= 500 else 6      # about 1 s .. 20 ms per pass
+    sample = OracleSample(args.workload, ORACLE_SAMPLE_LOG2[0] - shrink, ORACLE_SAMPLE_LOG2[1] - shrink)
     alg_bytes = full_algorithmic_bytes(args.workload)
     for _ in range(args.warmup):
         sample.run()
@@ -213,20 +276,114 @@ def run_reference(args):
         spent += s
     est = sum(ests) / len(ests)
     value = alg_bytes / est / 1e9
+    shape = FULL_SHAPE.get(args.workload)
+    if shape:
+        config = config_keys(args.workload, shape["n"], shape["k"], shape["k"], FULL_TRIALS.get(args.workload, 100), alg_bytes, 1)
+    else:
+        config = config_keys(args.workload, 1 << 24, 2048, 1024, 100, alg_bytes, 1)
+        config["step"] = config["step"].replace("2048 tensors", "about 2048 tensors")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "what": WORKLOAD_NOTES[args.workload],
-                   "note": "ms_per_step is the time of one full step estimated from the timed sample"},
+        "warmup": args.warmup, "ms_per_step": spent / max(1, args.steps) * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.description},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "gpu_launches": 0, "sample_seconds_per_step": spent / max(1, args.steps),
+        "gpu_launches": 0, "full_step_ms_estimate": est * 1e3,
+        "note": "each step is one pass over the bounded sample named in cpu_baseline.sample; ms_per_step is the measured "
+                "time of that pass, value = algorithmic bytes of a full step / full_step_ms_estimate",
     }
     print(json.dumps(line))
 
 
 # ----------------------------------------------------------------------------- GPU arm
+def _clone_population(pop):
+    refs = [r.clone() for r in pop.refs]
+    tensors = [workloads.Tensor(t.cand.clone(), t.ref_index, t.group, t.dtype) for t in pop.tensors]
+    return workloads.Population(pop.name, refs, tensors, pop.n_group, pop.atol, pop.rtol, pop.times, pop.base_times, pop.facts)
+
+
+def measure_config(evo, ctx, name, device, peak, reps):
+    """One of the smaller synthetic populations: device time of the main kernel alone, of the whole evo_validate call
+    (calls issued back to back) and of the whole step, all with CUDA events on the launching stream.
+    Populations that fit in L2 are labelled so; config 3 (272 MB, about twice L2) is run on three disjoint copies in
+    rotation so that no call finds its tensors in L2."""
+    pop = getattr(workloads, name)(device)
+    alg_bytes = pop.algorithmic_bytes()
+    copies = [pop] + ([_clone_population(pop), _clone_population(pop)] if name == "config3" else [])
+    preps, n_tensors = [], len(pop.tensors)
+    for p in copies:
+        preps.append(evo.Prepared([t.cand for t in p.tensors], [p.refs[t.ref_index] for t in p.tensors],
+                                  [t.group for t in p.tensors], p.n_group))
+    n_gen = gen_elems(pop)
+    gen_buf = torch.empty(n_gen, dtype=torch.float32, device=device)
+    results = torch.empty((n_tensors, 40), dtype=torch.uint8, device=device)
+    gpass = torch.empty(pop.n_group, dtype=torch.int32, device=device)
+    fits = torch.empty((pop.n_group, 16), dtype=torch.uint8, device=device)
+
+    def validate(i):
+        evo.evo_validate(preps[i % len(preps)], None, pop.atol, pop.rtol, results=results, group_pass=gpass, ctx=ctx)
+
+    def step(i):
+        evo.evo_gen_inputs(3000 + i, 0, evo.EVO_F32, n_gen, gen_buf, ctx=ctx)
+        validate(i)
+        evo.evo_fitness(pop.times, pop.base_times, gpass, out=fits, ctx=ctx)
+
+    def timed(fn):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(reps):
+            fn(i)
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    call_ms = timed(validate)
+    step_ms = timed(step)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in evs:
+        a.record()
+        b.record()
+    torch.cuda.synchronize()
+    for i, (a, b) in enumerate(evs):
+        ctx.set_timing_events(a, b)
+        validate(i)
+    torch.cuda.synchronize()
+    kernel_ms = statistics.median(a.elapsed_time(b) for a, b in evs)
+    fits_l2 = alg_bytes < 100 * (1 << 20)
+    out = {
+        "what": WORKLOAD_NOTES[name], "tensors": n_tensors, "candidates": pop.n_group, "algorithmic_bytes": alg_bytes,
+        "reps": reps, "kernel_ms": kernel_ms, "call_ms": call_ms, "step_ms": step_ms,
+        "kernel_gbs": alg_bytes / (kernel_ms * 1e-3) / 1e9, "call_gbs": alg_bytes / (call_ms * 1e-3) / 1e9,
+        "step_gbs": alg_bytes / (step_ms * 1e-3) / 1e9,
+        "kernel_frac_of_peak": alg_bytes / (kernel_ms * 1e-3) / 1e9 / peak, "step_frac_of_peak": alg_bytes / (step_ms * 1e-3) / 1e9 / peak,
+        "candidates_per_s": pop.n_group / (step_ms * 1e-3),
+        "memory": ("L2: the population fits in the 126 MB L2, the figures are not HBM rates" if fits_l2 else
+                   "L2 defeated: three disjoint copies of the population in rotation" if len(copies) > 1 else
+                   "inputs larger than L2"),
+        "kernel": "validate_pass1 (CUDA events around the launch, median)",
+        "call": "evo_validate, calls back to back (CUDA events around the loop)",
+    }
+    if name == "config5":
+        # load balance as measured: every CTA's own begin and end clock in one extra, untimed call
+        ctx.cta_timing(True)
+        validate(0)
+        t = ctx.read_cta_times()
+        ctx.cta_timing(False)
+        if len(t):
+            busy = (t[:, 1] - t[:, 0]).astype("float64")
+            out["load_balance"] = {"ctas": int(len(t)), "max_over_mean_cta_time": float(busy.max() / busy.mean()),
+                                   "min_over_mean_cta_time": float(busy.min() / busy.mean()),
+                                   "mean_cta_ms": float(busy.mean() * 1e-6),
+                                   "kernel_span_ms": float((t[:, 1].max() - t[:, 0].min()) * 1e-6),
+                                   "how": "%globaltimer at the start and the end of every persistent CTA of validate_pass1"}
+    del preps, copies, pop
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import paper_2510_03760_b200 as evo
 
@@ -369,30 +526,66 @@ def run_ours(args):
                 "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms_avg": kern_avg_ms,
                 "kernel_ms_min": min(kern_ms), "kernel_ms_max": max(kern_ms)}
 
-    cpu = None
+    roofline["datasheet_peak"] = DATASHEET_HBM_GBS
+    roofline["frac_of_datasheet"] = achieved / DATASHEET_HBM_GBS
+    roofline["note"] = ("frac is against the measured copy bandwidth of this pool's B200s (a read+write copy; a read-only stream "
+                        "can exceed it a little); frac_of_datasheet is against the nominal %d GB/s" % DATASHEET_HBM_GBS)
+
+    # the other synthetic populations, with the main one out of the way
+    config = config_keys(args.workload, n_gen, len(cands), n_group, int(pop.times.shape[1]), alg_bytes, world)
+    candidate_bytes = pop.candidate_bytes()
+    per_config = None
+    if args.per_config:
+        del prepared, cands, refs, pop, gen_buf
+        torch.cuda.empty_cache()
+        per_config = {}
+        for name, reps in (("config1", 200), ("config2", 200), ("config3", 100), ("config5", 20)):
+            if name != args.workload:
+                per_config[name] = measure_config(evo, ctx, name, device, peak, reps)
+
+    cpu = cpu_many = None
     if not args.no_cpu_baseline:
-        sample = OracleSample(args.workload, 28, 27)          # about 10-20 s of single-thread work
-        est, spent = sample.run()
-        cpu = {"value": alg_bytes / est / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample.description,
-               "seconds": spent, "host_cores_available": os.cpu_count()}
+        # about 10 s of single-thread work: the sample of the reference arm, several passes
+        sample = OracleSample(args.workload, ORACLE_SAMPLE_LOG2[0], ORACLE_SAMPLE_LOG2[1])
+        sample.run()
+        ests, spent, passes = [], 0.0, 0
+        while spent < 10.0 and passes < 64:
+            est, s_ = sample.run()
+            ests.append(est)
+            spent += s_
+            passes += 1
+        est = sum(ests) / len(ests)
+        cpu = {"value": alg_bytes / est / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": sample.description + "; %d passes" % passes, "seconds": spent,
+               "host_cores_available": len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()}
+        try:
+            cpu_many = oracle_many_processes(args.workload, alg_bytes, max(2, passes // 2))
+        except Exception as exc:        # a baseline leg must not take the benchmark line with it
+            cpu_many = {"value": None, "error": repr(exc)}
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "n_gpus_requested": args.gpus, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "what": WORKLOAD_NOTES[args.workload],
-                   "step": "evo_gen_inputs(%d fp32 normals) + evo_validate(%d tensors) + evo_fitness(%d x %d trials)"
-                           % (n_gen, len(cands), n_group, pop.times.shape[1]),
-                   "algorithmic_bytes_per_step": alg_bytes, "l2": "inputs larger than L2" if alg_bytes > (1 << 28) else "inputs fit in L2",
-                   "replicas": world},
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
         "candidates_per_s": cand_per_s, "frac_of_hbm_peak": value / world / peak,
-        "candidate_bytes_gbs": world * pop.candidate_bytes() / (ms_per_step * 1e-3) / 1e9, "plan": plan_info,
+        "frac_of_datasheet_hbm": value / world / DATASHEET_HBM_GBS,
+        "candidate_bytes_gbs": world * candidate_bytes / (ms_per_step * 1e-3) / 1e9, "plan": plan_info,
         "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roofline, "cpu_baseline": cpu,
+        "roofline": roofline, "cpu_baseline": cpu, "cpu_baseline_all_cores": cpu_many, "per_config": per_config,
     }
     print(json.dumps(line))
     if distributed:
         dist.destroy_process_group()
+
+
+def torchrun_command(n_gpus, argv):
+    """The command line `--gpus N` re-executes itself as when no launcher started it: N local ranks, one per GPU."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n_gpus),
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
 
 
 def main():
@@ -405,6 +598,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", dest="per_config", action="store_false",
+                    help="skip the figures of the other synthetic populations (configs 1, 2, 3, 5)")
     ap.add_argument("--log2-elems", type=int, default=None,
                     help="config4 only: shrink every tensor to 2^X elements (a small case for profiler captures; "
                          "not the benchmark configuration)")
@@ -414,6 +609,14 @@ def main():
             ap.error("--log2-elems needs --workload config4 and 12 <= X <= 28")
         args.no_cpu_baseline = True
         WORKLOAD_NOTES["config4"] = "REDUCED: 16 fp32 candidates x 2^%d elements sharing one reference" % args.log2_elems
+    if args.workload != "config4" or args.log2_elems is not None:
+        args.per_config = False
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        cmd = torchrun_command(args.gpus, sys.argv[1:])
+        os.execv(cmd[0], cmd)
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        ap.error("--gpus %d, but the launcher started %d rank(s)" % (args.gpus, world))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -28,6 +28,11 @@
  *     stream) only enqueue work; results are in device memory once the stream
  *     reaches that point.  The *_host variants synchronise the stream before they
  *     return.
+ *   - The kernels of a context's calls are launched so that each may begin its
+ *     set-up while the kernel before it in the stream is still running
+ *     (programmatic dependent launch); each waits for that kernel to complete
+ *     before it reads or writes any global memory, so stream order is kept for
+ *     every buffer.  evo_set_overlapped_launch(ctx, 0) turns this off.
  *   - A context owns a scratch workspace that grows on demand (cudaMalloc inside
  *     the call that needs it, never during stream capture by design of the
  *     caller) and is released by evo_destroy.  Use one context per stream; calls
@@ -350,9 +355,16 @@ EVO_API int evo_select_elite(evo_ctx* ctx, const evo_fit* fits /* device */, uin
  *   - The first call on each device looks up the scratch's device address (no allocation, but a
  *     runtime query): make that first call before starting any stream capture.
  *   - All calls on one device share the one scratch array.  It keeps whatever the previous call
- *     left; nothing in it needs clearing, since each call overwrites every word it later reads.
+ *     left.  The only word that must start at zero, the status word that a kernel raises when one
+ *     of its bounded waits runs out, is cleared on the stream at the head of every call; everything
+ *     else a call reads it has written itself.  So a call reports its own waits only: results
+ *     carry EVO_FLAG_INCOMPLETE (pass = 0) exactly when a wait of THAT call ran out, and the next
+ *     call starts clean - no restart and no extra call is needed to recover.
  *     But two calls whose kernels overlap on the GPU (different streams, or different threads)
  *     would overwrite each other's schedule: keep calls on one device ordered, e.g. on one stream.
+ *   - The schedule reaches the device as the arguments of small kernels (one launch per 16 KiB of
+ *     schedule, a few KiB for typical populations): the call hands the runtime no pointer into
+ *     host memory that it frees afterwards, and the host does not wait for the stream.
  *   - It calls no cudaMalloc, cudaFree, cudaMallocHost nor any other allocating CUDA routine.
  * evo_validate_static_error: message of the calling thread's last failing evo_validate_static
  * call ("" if it succeeded); static storage, never NULL.
@@ -389,8 +401,10 @@ EVO_API int evo_plan_inspect(const void* const* cand_ptrs, const void* ref_ptr, 
  * two CUDA events (cudaEvent_t passed as void*, created by the caller with timing enabled) on
  * its stream: `start` right before and `stop` right after the launch of the main checking
  * kernel (the first pass over the tensors).  The request is consumed by that call; pass NULLs
- * to cancel.  For measuring the kernel alone inside a longer stream of work.  (The paper has
- * no counterpart.)
+ * to cancel, and a call that fails consumes it too.  The small kernels before it (the store of
+ * the schedule, the warm start of the max d/|r| filter on short runs) lie outside the pair.
+ * For measuring the kernel alone inside a longer stream of work.  (The paper has no
+ * counterpart.)
  */
 EVO_API int evo_set_timing_events(evo_ctx* ctx, void* start, void* stop);
 
@@ -418,6 +432,26 @@ EVO_API int evo_selftest_wait(evo_ctx* ctx, uint32_t limit_us, void* stream);
 
 /* Number of kernels this context has launched so far (for accounting in benchmarks). */
 EVO_API uint64_t evo_launch_count(const evo_ctx* ctx);
+
+/*
+ * evo_set_overlapped_launch - turn programmatic dependent launch of the context's kernels on
+ * (default) or off.  Off, every kernel starts only after the work before it in the stream has
+ * finished, as with an ordinary launch.  (The paper has no counterpart.)
+ */
+EVO_API int evo_set_overlapped_launch(evo_ctx* ctx, int enable);
+
+/*
+ * evo_debug_cta_timing / evo_debug_read_cta_times - how evenly a population spreads over the
+ * persistent CTAs of evo_validate's main kernel, measured rather than planned.  While enabled,
+ * every CTA of that kernel writes the GPU's nanosecond clock (%globaltimer) when it starts
+ * working and when it is done, into a buffer of the context (allocated by the next
+ * evo_validate call).  evo_debug_read_cta_times waits for the device and copies the pairs
+ * (begin, end) of the last such call to `begin_end_ns` (host, 2 * capacity words; CTA b at
+ * 2b, 2b + 1); *n_ctas receives how many CTAs that call ran.  Meant for benchmarks; leave it
+ * off otherwise.  (The paper has no counterpart.)  Errors: EVO_ERR_ARG, EVO_ERR_CUDA.
+ */
+EVO_API int evo_debug_cta_timing(evo_ctx* ctx, int enable);
+EVO_API int evo_debug_read_cta_times(evo_ctx* ctx, uint64_t* begin_end_ns /* host */, uint32_t capacity, uint32_t* n_ctas /* host */);
 
 #ifdef __cplusplus
 }

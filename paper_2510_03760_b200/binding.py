@@ -67,6 +67,12 @@ def load_library():
     L.evo_check.restype = i32
     L.evo_selftest_wait.argtypes = [vp, u32, vp]
     L.evo_selftest_wait.restype = i32
+    L.evo_set_overlapped_launch.argtypes = [vp, i32]
+    L.evo_set_overlapped_launch.restype = i32
+    L.evo_debug_cta_timing.argtypes = [vp, i32]
+    L.evo_debug_cta_timing.restype = i32
+    L.evo_debug_read_cta_times.argtypes = [vp, vp, u32, vp]
+    L.evo_debug_read_cta_times.restype = i32
     L.evo_gen_inputs.argtypes = [vp, u64, u64, i32, u64, vp, vp]
     L.evo_gen_inputs.restype = i32
     for name in ("evo_validate", "evo_validate_host"):
@@ -128,6 +134,21 @@ class Context:
             self._h, C.c_void_p(start.cuda_event) if start is not None else None,
             C.c_void_p(stop.cuda_event) if stop is not None else None)
         self.check(st)
+
+    def set_overlapped_launch(self, enable):
+        """evo_set_overlapped_launch: programmatic dependent launch of this context's kernels on/off."""
+        self.check(load_library().evo_set_overlapped_launch(self._h, 1 if enable else 0))
+
+    def cta_timing(self, enable):
+        """evo_debug_cta_timing: have evo_validate's main kernel record each CTA's begin and end clock."""
+        self.check(load_library().evo_debug_cta_timing(self._h, 1 if enable else 0))
+
+    def read_cta_times(self, capacity=4096):
+        """evo_debug_read_cta_times: numpy uint64 array [n_ctas, 2] (begin, end) in ns of the last timed call."""
+        buf = np.zeros((int(capacity), 2), dtype=np.uint64)
+        n = C.c_uint32(0)
+        self.check(load_library().evo_debug_read_cta_times(self._h, C.c_void_p(buf.ctypes.data), int(capacity), C.byref(n)))
+        return buf[: min(int(n.value), int(capacity))]
 
     def synchronize(self, stream=None):
         """evo_check: wait for `stream` and raise EvoError(-6) if a device-side wait ran out."""

@@ -135,6 +135,7 @@ int evo_destroy(evo_ctx* ctx) {
     if (ctx->d_stage) (void)cudaFree(ctx->d_stage);
     if (ctx->d_feedback) (void)cudaFree(ctx->d_feedback);
     if (ctx->d_seeds) (void)cudaFree(ctx->d_seeds);
+    if (ctx->d_cta_times) (void)cudaFree(ctx->d_cta_times);
     if (ctx->d_small) (void)cudaFree(ctx->d_small);
     if (ctx->plan_consumed) (void)cudaEventDestroy(ctx->plan_consumed);
     delete ctx;
@@ -171,5 +172,30 @@ int evo_check(evo_ctx* ctx, void* stream) {
 }
 
 uint64_t evo_launch_count(const evo_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int evo_debug_cta_timing(evo_ctx* ctx, int enable) {
+    if (!ctx) return EVO_ERR_ARG;
+    ctx->cta_timing = enable != 0;
+    if (!ctx->cta_timing) ctx->cta_times_n = 0;
+    return EVO_OK;
+}
+
+int evo_debug_read_cta_times(evo_ctx* ctx, uint64_t* begin_end_ns, uint32_t capacity, uint32_t* n_ctas) {
+    if (!ctx || !n_ctas || (capacity > 0 && !begin_end_ns)) return EVO_ERR_ARG;
+    *n_ctas = ctx->cta_times_n;
+    const uint32_t n = ctx->cta_times_n < capacity ? ctx->cta_times_n : capacity;
+    if (n == 0) return EVO_OK;
+    evo::DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
+    EVO_CUDA_TRY(ctx, cudaDeviceSynchronize());
+    EVO_CUDA_TRY(ctx, cudaMemcpy(begin_end_ns, ctx->d_cta_times, static_cast<size_t>(n) * 16, cudaMemcpyDeviceToHost));
+    return EVO_OK;
+}
+
+int evo_set_overlapped_launch(evo_ctx* ctx, int enable) {
+    if (!ctx) return EVO_ERR_ARG;
+    ctx->pdl = enable != 0;
+    return EVO_OK;
+}
 
 }  // extern "C"

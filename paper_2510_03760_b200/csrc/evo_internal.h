@@ -26,6 +26,10 @@ struct evo_ctx {
     cudaEvent_t plan_consumed = nullptr;                       // the last plan upload has been read
     bool plan_in_flight = false;
     cudaEvent_t time_start = nullptr, time_stop = nullptr;     // one-shot request of evo_set_timing_events
+    bool pdl = true;                                           // launch kernels so that they may overlap their predecessor's tail
+    bool cta_timing = false;                                   // evo_debug_cta_timing: the first pass records per-CTA clocks
+    void* d_cta_times = nullptr; size_t d_cta_times_bytes = 0; // two 64-bit %globaltimer readings per CTA
+    uint32_t cta_times_n = 0;                                  // CTAs of the last timed first pass
 };
 
 namespace evo {
@@ -50,6 +54,32 @@ struct DeviceGuard {
 inline uint32_t* status_word(evo_ctx* ctx) { return reinterpret_cast<uint32_t*>(static_cast<char*>(ctx->d_small) + 128); }
 // Synchronises `stream`, then reads and clears the status word: EVO_OK or EVO_ERR_TIMEOUT.
 int sync_and_check(evo_ctx* ctx, cudaStream_t stream, const char* who);
+
+// Launches `kernel`; with `pdl` the launch carries the programmatic-stream-serialization
+// attribute, so the kernel may begin (up to its griddepcontrol.wait) while the kernel before it
+// in the stream is still running.  If a launch with the attribute is refused, it is repeated
+// without.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl,
+                          const Args&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    if (e != cudaSuccess && pdl) {
+        (void)cudaGetLastError();
+        cfg.numAttrs = 0;
+        e = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    }
+    return e;
+}
 
 inline size_t elem_bytes(int dtype) { return dtype == EVO_F16 || dtype == EVO_BF16 ? 2 : 4; }
 

@@ -87,26 +87,36 @@ __device__ RowMedian warp_statistic(const float* row, uint32_t m, int stat, uint
     return RowMedian{med, 1u};
 }
 
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
-fitness_kernel(const float* __restrict__ times, uint64_t n_rows, uint32_t trials, int stat, uint32_t warmup, uint32_t trim,
-               const RowMedian* __restrict__ base /* nullptr: write the row's statistic to base_out */,
-               RowMedian* __restrict__ base_out, const uint32_t* __restrict__ pass, evo_fit* __restrict__ out) {
+// One launch: warps 0..3 of a CTA take one row of candidate times each, warp 4 takes the
+// baseline row (every CTA computes the baseline's statistic again: a hundred floats, cheaper
+// than a launch of its own and a dependency on it).
+__global__ void __launch_bounds__((kWarpsPerCta + 1) * 32)
+fitness_kernel(const float* __restrict__ times, uint64_t n_rows, uint32_t trials, const float* __restrict__ base_times,
+               uint32_t base_trials, int stat, uint32_t warmup, uint32_t trim, const uint32_t* __restrict__ pass,
+               evo_fit* __restrict__ out) {
     extern __shared__ float smem[];
+    __shared__ RowMedian s_base;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // the verdicts in `pass` come from the kernel before
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t m = trials - warmup;                                   // runs that count
-    const uint32_t per_warp = (stat == EVO_STAT_TRIMMED_MEAN ? 2 * m : m) + 2;
-    float* row = smem + static_cast<size_t>(warp) * per_warp;
+    const bool is_base = warp == kWarpsPerCta;
+    const uint32_t m = (is_base ? base_trials : trials) - warmup;            // runs that count
+    const uint32_t per_row = (stat == EVO_STAT_TRIMMED_MEAN ? 2 * (trials - warmup) : trials - warmup) + 2;
+    float* row = smem + static_cast<size_t>(warp) * per_row;                 // the baseline's area comes last
     float* slot = row + m;
     float* sorted = slot + 2;
     const uint64_t r = static_cast<uint64_t>(blockIdx.x) * kWarpsPerCta + warp;
-    if (r >= n_rows) return;
-    const float* src = times + r * trials + warmup;
-    for (uint32_t i = lane; i < m; i += 32) row[i] = src[i];
-    __syncwarp();
-    const RowMedian med = warp_statistic(row, m, stat, trim, lane, slot, sorted);
-    if (lane != 0) return;
-    if (!base) { *base_out = med; return; }
-    const RowMedian b = *base;
+    RowMedian med{0.f, 0u};
+    if (is_base || r < n_rows) {
+        const float* src = (is_base ? base_times : times + r * trials) + warmup;
+        for (uint32_t i = lane; i < m; i += 32) row[i] = src[i];
+        __syncwarp();
+        med = warp_statistic(row, m, stat, trim, lane, slot, sorted);
+        if (is_base && lane == 0) s_base = med;
+    }
+    __syncthreads();
+    if (is_base || r >= n_rows || lane != 0) return;
+    const RowMedian b = s_base;
     evo_fit f;
     f.median_ms = med.ok ? med.median : 0.f;
     f.speedup = 0.f;
@@ -119,29 +129,23 @@ fitness_kernel(const float* __restrict__ times, uint64_t n_rows, uint32_t trials
     out[r] = f;
 }
 
-size_t smem_bytes(uint32_t trials, int stat, uint32_t warmup) {
+size_t row_floats(uint32_t trials, int stat, uint32_t warmup) {
     const size_t m = trials - warmup;
-    return ((stat == EVO_STAT_TRIMMED_MEAN ? 2 * m : m) + 2) * sizeof(float) * kWarpsPerCta;
+    return (stat == EVO_STAT_TRIMMED_MEAN ? 2 * m : m) + 2;
 }
 
 int fitness_device(evo_ctx* ctx, const float* times, uint64_t n_cand, uint32_t trials, const float* base_times,
                    uint32_t base_trials, const uint32_t* pass, int stat, uint32_t warmup, uint32_t trim, evo_fit* out,
                    cudaStream_t stream) {
-    RowMedian* d_base = static_cast<RowMedian*>(ctx->d_small);
-    const size_t smem_base = smem_bytes(base_trials, stat, warmup), smem_rows = smem_bytes(trials, stat, warmup);
-    if (std::max(smem_base, smem_rows) > 48 * 1024)
-        EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(fitness_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               static_cast<int>(smem_bytes(kMaxTrials, EVO_STAT_TRIMMED_MEAN, 0))));
-    fitness_kernel<<<1, kWarpsPerCta * 32, smem_base, stream>>>(base_times, 1, base_trials, stat, warmup, trim, nullptr, d_base,
-                                                               nullptr, nullptr);
-    ctx->launches += 1;
-    EVO_CUDA_TRY(ctx, cudaGetLastError());
     if (n_cand == 0) return EVO_OK;
+    const size_t smem = (kWarpsPerCta * row_floats(trials, stat, warmup) + row_floats(base_trials, stat, warmup)) * sizeof(float);
+    if (smem > 48 * 1024)
+        EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(fitness_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>((kWarpsPerCta + 1) * row_floats(kMaxTrials, EVO_STAT_TRIMMED_MEAN, 0) * sizeof(float))));
     const unsigned grid = static_cast<unsigned>((n_cand + kWarpsPerCta - 1) / kWarpsPerCta);
-    fitness_kernel<<<grid, kWarpsPerCta * 32, smem_rows, stream>>>(times, n_cand, trials, stat, warmup, trim, d_base, nullptr,
-                                                                  pass, out);
+    EVO_CUDA_TRY(ctx, evo::launch(fitness_kernel, dim3(grid), dim3((kWarpsPerCta + 1) * 32), smem, stream, ctx->pdl, times, n_cand,
+                                  trials, base_times, base_trials, stat, warmup, trim, pass, out));
     ctx->launches += 1;
-    EVO_CUDA_TRY(ctx, cudaGetLastError());
     return EVO_OK;
 }
 

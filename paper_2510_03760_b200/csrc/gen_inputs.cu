@@ -73,6 +73,9 @@ template <int DT, bool VEC>
 __global__ void __launch_bounds__(256) gen_kernel(const __grid_constant__ RoundKeys rk, uint64_t first_block, uint64_t n_blocks,
                                                   uint32_t lead, uint64_t n, typename Out<DT>::T* __restrict__ out) {
     using T = typename Out<DT>::T;
+    // may start while the kernel before it in the stream still runs; `out` is not written before that one is done
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
     for (uint64_t j = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < n_blocks; j += stride) {
         const uint4 w = philox4x32_10(first_block + j, rk);
@@ -107,10 +110,9 @@ cudaError_t launch(evo_ctx* ctx, uint64_t seed, uint64_t offset, uint64_t n, voi
     const uint64_t cap = static_cast<uint64_t>(ctx->sm_count) * 8 * 4;   // a few waves of 8 resident CTAs per SM
     const unsigned grid = static_cast<unsigned>(want < cap ? want : cap);
     const RoundKeys rk = round_keys(seed);
-    if (vec) gen_kernel<DT, true><<<grid, 256, 0, stream>>>(rk, offset >> 2, n_blocks, lead, n, static_cast<T*>(out));
-    else     gen_kernel<DT, false><<<grid, 256, 0, stream>>>(rk, offset >> 2, n_blocks, lead, n, static_cast<T*>(out));
     ctx->launches += 1;
-    return cudaGetLastError();
+    if (vec) return evo::launch(gen_kernel<DT, true>, dim3(grid), dim3(256), 0, stream, ctx->pdl, rk, offset >> 2, n_blocks, lead, n, static_cast<T*>(out));
+    return evo::launch(gen_kernel<DT, false>, dim3(grid), dim3(256), 0, stream, ctx->pdl, rk, offset >> 2, n_blocks, lead, n, static_cast<T*>(out));
 }
 
 }  // namespace

@@ -49,8 +49,9 @@ namespace {
 using namespace evo;
 
 constexpr int kCtasPerSm = 2;
-constexpr int kStages = 6;                          // ring depth per CTA
-constexpr int kStageBytes = kTileElems * 4;         // 16 KiB: one fp32 tile (a 16-bit tile uses half)
+constexpr int kStages = 12;                         // ring depth per CTA
+constexpr int kStageBytes = kTileElems * 2;         // 8 KiB: one 16-bit tile; an fp32 tile travels as two stages
+constexpr int kStageVecs = kStageBytes / (16 * kThreads);   // 16-byte vectors per consumer thread and stage (2)
 constexpr size_t kRingBytes = static_cast<size_t>(kStages) * kStageBytes;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, then give up
 constexpr uint64_t kSeedBelowTilesPerCta = 32;               // runs shorter than this get the seed pass
@@ -111,6 +112,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar), "l"(pol) : "memory");
 }
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+
+// Programmatic dependent launch.  Every kernel of a call is launched so that it may start while
+// its predecessor in the stream is still running: it does its set-up, then waits here until the
+// predecessor has completed and its writes are visible, and only then touches global memory.
+// Every kernel waits (even one that needs nothing from its predecessor), so completion stays
+// transitive along the stream.  Launched without the attribute, both are no-ops.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ float rcp_approx(float x) {
     float y;
@@ -228,6 +237,24 @@ __device__ __forceinline__ void ring_release(Ring& g, int lane) {
     g.advance();
 }
 
+// One tile (kTileElems elements of one tensor) out of the ring into registers: it arrives as one
+// stage (16-bit types) or two consecutive stages (fp32); thread t's vector v is vector
+// (v mod kStageVecs) * kThreads + t of stage v / kStageVecs.  Each stage is handed back as soon
+// as the warp has its share.  False if a wait ran out.
+template <int DT>
+__device__ __forceinline__ bool take_tile(Ring& g, uint4 (&v)[Elem<DT>::kVecs], int lane) {
+    constexpr uint32_t kVecStride = kThreads * 16;
+#pragma unroll
+    for (int p = 0; p < Elem<DT>::kVecs / kStageVecs; ++p) {
+        if (!ring_acquire(g)) return false;
+        const uint32_t a = g.data() + threadIdx.x * 16;
+#pragma unroll
+        for (int q = 0; q < kStageVecs; ++q) v[p * kStageVecs + q] = lds128(a + q * kVecStride);
+        ring_release(g, lane);
+    }
+    return true;
+}
+
 // IEEE division, kept out of line: the walks below name it at 16 unrolled positions and run it
 // at one or two of them, so its body would only bloat the hot loop's instruction footprint.
 __device__ __noinline__ float div_rn(float a, float b) { return __fdiv_rn(a, b); }
@@ -251,19 +278,15 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
                                           uint32_t* s_mr, const void* const* s_cand, Ring& g, int warp, int lane) {
     using E = Elem<DT>;
     if (g.dead) return;
-    constexpr uint32_t kVecStride = kThreads * 16;
     float r[kEpt];
-    if (!ring_acquire(g)) return;
     {
-        const uint32_t a = g.data() + threadIdx.x * 16;
+        uint4 rv[E::kVecs];
+        if (!take_tile<DT>(g, rv, lane)) return;
 #pragma unroll
-        for (int v = 0; v < E::kVecs; ++v) {
-            const uint4 x = lds128(a + v * kVecStride);
+        for (int v = 0; v < E::kVecs; ++v)
 #pragma unroll
-            for (int e = 0; e < E::kPerVec; ++e) r[v * E::kPerVec + e] = E::at(x, e);
-        }
+            for (int e = 0; e < E::kPerVec; ++e) r[v * E::kPerVec + e] = E::at(rv[v], e);
     }
-    ring_release(g, lane);
     // The smallest tolerance among this thread's 16 reference elements: tol = atol + rtol*|r| does not decrease
     // with |r| (each rounding is monotone), so it is the tolerance of the smallest |r|.  A member whose largest
     // difference over these elements stays within it has no mismatch here, and none is counted element by element.
@@ -274,14 +297,8 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
     const uint64_t vec0 = t * (kTileElems / E::kPerVec) + threadIdx.x;   // this thread's first vector of the tile
 #pragma unroll 1
     for (int k = 0; k < K; ++k) {
-        if (!ring_acquire(g)) return;
         uint4 cv[E::kVecs];
-        {
-            const uint32_t a = g.data() + threadIdx.x * 16;
-#pragma unroll
-            for (int v = 0; v < E::kVecs; ++v) cv[v] = lds128(a + v * kVecStride);
-        }
-        ring_release(g, lane);
+        if (!take_tile<DT>(g, cv, lane)) return;
         Acc* acc = &s_acc[k][warp];
         // Running maximum of d/|r| of this member, shared by the CTA's warps.  A stale (smaller)
         // value only makes the filter fire more often.
@@ -404,6 +421,26 @@ __device__ __noinline__ void slow_tile(const SetRec& S, uint64_t t, float atol, 
     }
 }
 
+// The whole vectors of a ragged last tile: only the stages that hold some of its `valid_vecs`
+// vectors were copied (the producer counts the same way); vectors that do not exist read as zero.
+template <int DT>
+__device__ __forceinline__ bool take_tail(Ring& g, uint4 (&v)[Elem<DT>::kVecs], uint32_t valid_vecs, int lane) {
+    constexpr uint32_t kVecStride = kThreads * 16;
+#pragma unroll
+    for (int p = 0; p < Elem<DT>::kVecs / kStageVecs; ++p) {
+#pragma unroll
+        for (int q = 0; q < kStageVecs; ++q) v[p * kStageVecs + q] = make_uint4(0u, 0u, 0u, 0u);
+        if (static_cast<uint32_t>(p) * kStageVecs * kThreads >= valid_vecs) continue;      // uniform for the CTA
+        if (!ring_acquire(g)) return false;
+        const uint32_t a = g.data() + threadIdx.x * 16;
+#pragma unroll
+        for (int q = 0; q < kStageVecs; ++q)
+            if ((p * kStageVecs + q) * kThreads + threadIdx.x < valid_vecs) v[p * kStageVecs + q] = lds128(a + q * kVecStride);
+        ring_release(g, lane);
+    }
+    return true;
+}
+
 // The ragged last tile of an aligned tensor.  Its whole 16-byte vectors (`valid_vecs` of
 // them) come through the ring like a full tile; a thread takes the same vectors as in
 // fast_tile but only those that exist, and applies the exact rule to each element.  Once per
@@ -414,20 +451,11 @@ template <int DT>
 __device__ __noinline__ uint32_t tail_tile(uint32_t n_members, uint32_t valid_vecs, float atol, float rtol,
                                            Acc (*s_acc)[kWarps], Ring g, int warp, int lane) {
     using E = Elem<DT>;
-    constexpr uint32_t kVecStride = kThreads * 16;
     uint4 rv[E::kVecs];
-    if (ring_acquire(g)) {
-        const uint32_t a = g.data() + threadIdx.x * 16;
-#pragma unroll
-        for (int v = 0; v < E::kVecs; ++v) rv[v] = lds128(a + v * kVecStride);
-        ring_release(g, lane);
+    if (take_tail<DT>(g, rv, valid_vecs, lane)) {
         for (uint32_t k = 0; k < n_members; ++k) {
-            if (!ring_acquire(g)) break;
             uint4 cv[E::kVecs];
-            const uint32_t b = g.data() + threadIdx.x * 16;
-#pragma unroll
-            for (int v = 0; v < E::kVecs; ++v) cv[v] = lds128(b + v * kVecStride);
-            ring_release(g, lane);
+            if (!take_tail<DT>(g, cv, valid_vecs, lane)) break;
             Lane st;
 #pragma unroll
             for (int v = 0; v < E::kVecs; ++v) {
@@ -559,21 +587,25 @@ __device__ __forceinline__ uint32_t producer_loop(const SetRec* __restrict__ set
         for (uint64_t t = t0; t < t1 && !g.dead; ++t) {
             const unsigned long long off = t * full_bytes;
             const uint32_t tile_bytes = t < sp.full_tiles ? full_bytes : sp.tail_vecs * 16u;
-            for (uint32_t j = 0; j <= S.k; ++j) {
+            for (uint32_t j = 0; j <= S.k && !g.dead; ++j) {
                 const unsigned long long base = __shfl_sync(full, mine, j == 0 ? 0 : static_cast<int>(j - 1));
                 const unsigned long long src = (j == 0 ? ref : base) + off;
-                int ok = 1;
-                if (lane == 0) {
-                    ok = mbar_wait(g.empty(), g.phase ^ 1u, g.abort_flag) ? 1 : 0;
-                    if (ok) {
-                        mbar_arrive_expect_tx(g.full(), tile_bytes);
-                        bulk_load(g.data(), reinterpret_cast<const void*>(src), tile_bytes, g.full(), pol);
+                // the tile in pieces of one stage each (one piece for 16-bit types, two for fp32, the last maybe short)
+                for (uint32_t done = 0; done < tile_bytes; done += kStageBytes) {
+                    const uint32_t piece = tile_bytes - done < static_cast<uint32_t>(kStageBytes) ? tile_bytes - done : kStageBytes;
+                    int ok = 1;
+                    if (lane == 0) {
+                        ok = mbar_wait(g.empty(), g.phase ^ 1u, g.abort_flag) ? 1 : 0;
+                        if (ok) {
+                            mbar_arrive_expect_tx(g.full(), piece);
+                            bulk_load(g.data(), reinterpret_cast<const void*>(src + done), piece, g.full(), pol);
+                        }
                     }
+                    ok = __shfl_sync(full, ok, 0);
+                    if (!ok) { g.dead = true; break; }
+                    g.advance();
+                    ++issued;
                 }
-                ok = __shfl_sync(full, ok, 0);
-                if (!ok) { g.dead = true; break; }
-                g.advance();
-                ++issued;
             }
         }
     }
@@ -583,14 +615,14 @@ __device__ __forceinline__ uint32_t producer_loop(const SetRec* __restrict__ set
 __global__ void __launch_bounds__(kBlock, kCtasPerSm)
 validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
                const CtaRange* __restrict__ ranges, Acc* __restrict__ partials, float atol, float rtol,
-               uint32_t* __restrict__ status, const uint32_t* __restrict__ seeds /* optional: see seed_kernel */) {
+               uint32_t* __restrict__ status, const uint32_t* __restrict__ seeds /* optional: see seed_kernel */,
+               unsigned long long* __restrict__ cta_times /* optional: %globaltimer at start and end of every CTA */) {
     extern __shared__ __align__(128) unsigned char s_ring[];
     __shared__ Acc s_acc[kMaxK][kWarps];
     __shared__ const void* s_cand[kMaxK];
     __shared__ uint32_t s_mr[kMaxK];         // per member: running maximum of d/|r| found on the fast path (bit pattern)
     __shared__ __align__(8) unsigned long long s_full[kStages], s_empty[kStages];
     __shared__ int s_abort;
-    const CtaRange rg = ranges[blockIdx.x];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) {
@@ -601,6 +633,11 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
         mbar_fence_init();
     }
     __syncthreads();
+    // Up to here nothing depended on earlier work in the stream; the plan, the seeds and the tensors do.
+    grid_dependents_may_launch();
+    grid_dependency_wait();
+    if (cta_times && threadIdx.x == 0) cta_times[2 * blockIdx.x] = global_ns();
+    const CtaRange rg = ranges[blockIdx.x];
     Ring g;
     g.full0 = smem_u32(&s_full[0]);
     g.empty0 = smem_u32(&s_empty[0]);
@@ -659,6 +696,7 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
         }
         if (threadIdx.x == 0) atomicOr(status, 1u);
     }
+    if (cta_times && threadIdx.x == 0) cta_times[2 * blockIdx.x + 1] = global_ns();
 }
 
 // Warm start for the filter of max d/|r|.  A CTA that begins a run knows no maximum for its
@@ -671,6 +709,8 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
 __global__ void __launch_bounds__(kThreads)
 seed_kernel(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members, uint32_t* __restrict__ seeds) {
     __shared__ uint32_t s_max[kWarps];
+    grid_dependents_may_launch();
+    grid_dependency_wait();
     const MemberRec M = members[blockIdx.x];
     const SetRec S = sets[M.set];
     const uint32_t n = static_cast<uint32_t>(S.n < static_cast<uint64_t>(kTileElems) ? S.n : static_cast<uint64_t>(kTileElems));
@@ -706,13 +746,37 @@ seed_kernel(const SetRec* __restrict__ sets, const MemberRec* __restrict__ membe
 // One warp per tensor: fold the partial records of the CTAs [cta_first, cta_last] in a
 // fixed order (lane-strided, then a xor tree).  If the first pass gave up on a wait, the
 // records are incomplete: every result then says so instead of carrying numbers.
-__global__ void __launch_bounds__(kThreads)
+// `fused` (a single CTA holds every tensor: small populations) also takes the candidate
+// verdicts afterwards, which saves a launch where launches are all the time there is.
+struct VerdictArgs { const uint32_t* offsets; const uint32_t* desc_of; uint32_t n_group; uint32_t* group_pass; };
+
+__device__ __forceinline__ void fold_partials(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
+                                              const CtaRange* __restrict__ ranges, const Acc* __restrict__ partials,
+                                              uint32_t m, int lane, evo_result* __restrict__ results,
+                                              const uint32_t* __restrict__ status);
+
+__global__ void __launch_bounds__(1024)
 validate_pass2(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
                const CtaRange* __restrict__ ranges, const Acc* __restrict__ partials,
-               uint32_t n_members, evo_result* __restrict__ results, const uint32_t* __restrict__ status) {
-    const uint32_t m = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (m >= n_members) return;
+               uint32_t n_members, evo_result* __restrict__ results, const uint32_t* __restrict__ status,
+               bool fused, VerdictArgs va) {
+    grid_dependents_may_launch();
+    grid_dependency_wait();
+    const uint32_t m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (m < n_members) fold_partials(sets, members, ranges, partials, m, threadIdx.x & 31, results, status);
+    if (!fused) return;
+    __syncthreads();              // the CTA's own writes to results[] are visible to it from here on
+    for (uint32_t g = threadIdx.x; g < va.n_group; g += blockDim.x) {
+        uint32_t ok = 1;
+        for (uint32_t i = va.offsets[g]; i < va.offsets[g + 1]; ++i) ok &= results[va.desc_of[i]].pass;
+        va.group_pass[g] = ok;
+    }
+}
+
+__device__ __forceinline__ void fold_partials(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
+                                              const CtaRange* __restrict__ ranges, const Acc* __restrict__ partials,
+                                              uint32_t m, int lane, evo_result* __restrict__ results,
+                                              const uint32_t* __restrict__ status) {
     const MemberRec M = members[m];
     if (*status != 0) {
         if (lane == 0) {
@@ -757,11 +821,26 @@ validate_pass2(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
 // Candidate verdicts: AND over the tensors of each candidate id.
 __global__ void group_verdict(const uint32_t* __restrict__ offsets, const uint32_t* __restrict__ desc_of,
                               const evo_result* __restrict__ results, uint32_t n_group, uint32_t* __restrict__ group_pass) {
+    grid_dependents_may_launch();
+    grid_dependency_wait();
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= n_group) return;
     uint32_t ok = 1;
     for (uint32_t i = offsets[g]; i < offsets[g + 1]; ++i) ok &= results[desc_of[i]].pass;
     group_pass[g] = ok;
+}
+
+// Small plans travel as kernel arguments: this kernel writes one chunk of a packed plan to its
+// place in device memory.  No staging buffer on the host, no copy engine, nothing the host has
+// to wait for before it may build the next plan; the launch itself carries the bytes.
+constexpr uint32_t kPlanChunkBytes = 16 * 1024;
+struct PlanChunk { uint4 w[kPlanChunkBytes / 16]; };
+__global__ void __launch_bounds__(256)
+plan_store(const __grid_constant__ PlanChunk chunk, uint4* __restrict__ dst, uint32_t n_vec, uint32_t* __restrict__ clear_word) {
+    grid_dependents_may_launch();
+    grid_dependency_wait();
+    for (uint32_t i = threadIdx.x; i < n_vec; i += blockDim.x) dst[i] = chunk.w[i];
+    if (clear_word && threadIdx.x == 0) *clear_word = 0u;
 }
 
 // Self-test of the bounded wait: one warp waits on a barrier that nothing will ever complete,
@@ -786,9 +865,119 @@ __global__ void wait_selftest_kernel(unsigned long long limit_ns, uint32_t* __re
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Where the parts of a packed plan sit, as byte offsets from the start of the plan area.
+struct PlanLayout { size_t o_sets, o_members, o_ranges, o_goff, o_gdesc, bytes; };
+
+PlanLayout layout_of(const Plan& plan, size_t first) {
+    PlanLayout L;
+    L.o_sets = first;
+    L.o_members = align_up(L.o_sets + plan.sets.size() * sizeof(SetRec), 256);
+    L.o_ranges = align_up(L.o_members + plan.members.size() * sizeof(MemberRec), 256);
+    L.o_goff = align_up(L.o_ranges + plan.ranges.size() * sizeof(CtaRange), 256);
+    L.o_gdesc = align_up(L.o_goff + plan.group_off.size() * 4, 256);
+    L.bytes = align_up(L.o_gdesc + plan.group_desc.size() * 4, 256);
+    return L;
+}
+
+// Packs the plan into `dst`, whose first byte stands for offset `first` of the layout.
+void pack_plan(const Plan& plan, const PlanLayout& L, size_t first, unsigned char* dst) {
+    auto put = [&](size_t o, const void* src, size_t bytes) { if (bytes) std::memcpy(dst + (o - first), src, bytes); };
+    put(L.o_sets, plan.sets.data(), plan.sets.size() * sizeof(SetRec));
+    put(L.o_members, plan.members.data(), plan.members.size() * sizeof(MemberRec));
+    put(L.o_ranges, plan.ranges.data(), plan.ranges.size() * sizeof(CtaRange));
+    put(L.o_goff, plan.group_off.data(), plan.group_off.size() * 4);
+    put(L.o_gdesc, plan.group_desc.data(), plan.group_desc.size() * 4);
+}
+
+// `bytes` of a packed plan from host memory to `dst` on the device as the arguments of one
+// plan_store launch per chunk (16-byte granules; dst is 16-byte aligned).  The first chunk may
+// also clear a word (the status word of a caller that has no other moment to do so).
+cudaError_t store_plan(const unsigned char* src, size_t bytes, unsigned char* dst, uint32_t* clear_word, bool pdl,
+                       cudaStream_t stream, uint64_t* launches) {
+    PlanChunk chunk;
+    size_t done = 0;
+    do {
+        const size_t piece = std::min<size_t>(bytes - done, kPlanChunkBytes);
+        if (piece) std::memcpy(chunk.w, src + done, piece);
+        const uint32_t n_vec = static_cast<uint32_t>((piece + 15) / 16);
+        const cudaError_t e = evo::launch(plan_store, dim3(1), dim3(256), 0, stream, pdl, chunk,
+                                          reinterpret_cast<uint4*>(dst + done), n_vec, done == 0 ? clear_word : nullptr);
+        if (e != cudaSuccess) return e;
+        if (launches) *launches += 1;
+        done += piece;
+    } while (done < bytes);
+    return cudaSuccess;
+}
+
+// Everything a call launches once its plan is in device memory: seed pass (optional), first
+// pass, second pass, verdicts.  Shared by the context-based and the allocation-free entry points.
+struct ChainArgs {
+    const unsigned char* d_plan;      // device address of layout offset 0
+    PlanLayout L;
+    Acc* d_parts;
+    uint32_t* d_status;
+    uint32_t* d_seeds;                // nullptr: no seed pass
+    unsigned long long* d_cta_times;  // nullptr: no per-CTA clock readings
+    float atol, rtol;
+    evo_result* results;
+    uint32_t* group_pass;
+    uint64_t n_group;
+    bool pdl;
+    cudaEvent_t ev_start, ev_stop;    // optional: around the first pass
+};
+
+cudaError_t launch_chain(const Plan& plan, const ChainArgs& a, cudaStream_t stream, uint64_t* launches) {
+    const SetRec* d_sets = reinterpret_cast<const SetRec*>(a.d_plan + a.L.o_sets);
+    const MemberRec* d_members = reinterpret_cast<const MemberRec*>(a.d_plan + a.L.o_members);
+    const CtaRange* d_ranges = reinterpret_cast<const CtaRange*>(a.d_plan + a.L.o_ranges);
+    const uint32_t* d_goff = reinterpret_cast<const uint32_t*>(a.d_plan + a.L.o_goff);
+    const uint32_t* d_gdesc = reinterpret_cast<const uint32_t*>(a.d_plan + a.L.o_gdesc);
+    const uint32_t n_members = static_cast<uint32_t>(plan.members.size());
+    const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
+    cudaError_t e;
+    auto count = [&]() { if (launches) *launches += 1; };
+    if (a.d_seeds && n_members > 0) {
+        e = evo::launch(seed_kernel, dim3(n_members), dim3(kThreads), 0, stream, a.pdl, d_sets, d_members, a.d_seeds);
+        if (e != cudaSuccess) return e;
+        count();
+    }
+    if (a.ev_start && (e = cudaEventRecord(a.ev_start, stream)) != cudaSuccess) return e;
+    if (n_ctas > 0) {
+        e = evo::launch(validate_pass1, dim3(n_ctas), dim3(kBlock), kRingBytes, stream, a.pdl, d_sets, d_members, d_ranges,
+                        a.d_parts, a.atol, a.rtol, a.d_status, static_cast<const uint32_t*>(a.d_seeds && n_members ? a.d_seeds : nullptr),
+                        a.d_cta_times);
+        if (e != cudaSuccess) return e;
+        count();
+    }
+    if (a.ev_stop && (e = cudaEventRecord(a.ev_stop, stream)) != cudaSuccess) return e;
+    // Up to 32 tensors: one CTA, one warp per tensor, takes the second pass and then the verdicts.
+    const bool fused = a.group_pass != nullptr && n_members <= 32;
+    VerdictArgs va{d_goff, d_gdesc, static_cast<uint32_t>(a.n_group), a.group_pass};
+    if (n_members > 0 || fused) {
+        const uint32_t block = fused ? std::max<uint32_t>(32u, 32u * n_members) : static_cast<uint32_t>(kThreads);
+        const uint32_t grid = fused ? 1u : (n_members + kWarps - 1) / kWarps;
+        e = evo::launch(validate_pass2, dim3(grid), dim3(block), 0, stream, a.pdl, d_sets, d_members, d_ranges,
+                        static_cast<const Acc*>(a.d_parts), n_members, a.results, static_cast<const uint32_t*>(a.d_status), fused, va);
+        if (e != cudaSuccess) return e;
+        count();
+    }
+    if (a.group_pass && !fused) {
+        e = evo::launch(group_verdict, dim3(static_cast<unsigned>((a.n_group + 255) / 256)), dim3(256), 0, stream, a.pdl, d_goff,
+                        d_gdesc, static_cast<const evo_result*>(a.results), static_cast<uint32_t>(a.n_group), a.group_pass);
+        if (e != cudaSuccess) return e;
+        count();
+    }
+    return cudaSuccess;
+}
+
+constexpr size_t kPlanAsArgumentsLimit = 2 * kPlanChunkBytes;      // larger plans go up with a copy from pinned memory
+
 int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs,
                     uint64_t n_desc, int dtype, float atol, float rtol, evo_result* results,
                     uint32_t* group_pass, uint64_t n_group, cudaStream_t stream, const char* who) {
+    // the one-shot timing request belongs to this call, whether it succeeds or not
+    const cudaEvent_t ev_start = ctx->time_start, ev_stop = ctx->time_stop;
+    ctx->time_start = ctx->time_stop = nullptr;
     if (n_desc > 0 && !results) return evo::fail(ctx, EVO_ERR_ARG, "%s: results must not be NULL", who);
     Plan plan;
     std::string err;
@@ -800,87 +989,63 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     evo::DeviceGuard guard(ctx->device);
     if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
 
-    // ---- pack and upload the plan ----
-    const size_t o_sets = 0;
-    const size_t o_members = align_up(o_sets + plan.sets.size() * sizeof(SetRec), 256);
-    const size_t o_ranges = align_up(o_members + plan.members.size() * sizeof(MemberRec), 256);
-    const size_t o_goff = align_up(o_ranges + plan.ranges.size() * sizeof(CtaRange), 256);
-    const size_t o_gdesc = align_up(o_goff + plan.group_off.size() * 4, 256);
-    const size_t plan_bytes = align_up(o_gdesc + plan.group_desc.size() * 4, 256) + 256;
-    st = evo::reserve_pinned(ctx, &ctx->h_plan, &ctx->h_plan_bytes, plan_bytes);
-    if (st != EVO_OK) return st;
-    st = evo::reserve_device(ctx, &ctx->d_plan, &ctx->d_plan_bytes, plan_bytes);
+    const PlanLayout L = layout_of(plan, 0);
+    st = evo::reserve_device(ctx, &ctx->d_plan, &ctx->d_plan_bytes, L.bytes + 256);
     if (st != EVO_OK) return st;
     st = evo::reserve_device(ctx, &ctx->d_partials, &ctx->d_partials_bytes, std::max<size_t>(plan.n_parts, 1) * sizeof(Acc));
     if (st != EVO_OK) return st;
     // Short runs (few tiles per CTA and member): seed the filter of max d/|r| first, see seed_kernel.
     // (Not for populations with fewer tiles than CTAs: those are bound by launch latency, which a further
     // kernel only adds to.)
-    const bool seed = plan.total_tiles >= max_ctas && plan.total_tiles / max_ctas < kSeedBelowTilesPerCta;
+    const bool seed = plan.total_tiles >= max_ctas && plan.total_tiles / max_ctas < kSeedBelowTilesPerCta && n_desc > 0;
     if (seed) {
-        st = evo::reserve_device(ctx, &ctx->d_seeds, &ctx->d_seeds_bytes, std::max<size_t>(n_desc, 1) * sizeof(uint32_t));
+        st = evo::reserve_device(ctx, &ctx->d_seeds, &ctx->d_seeds_bytes, n_desc * sizeof(uint32_t));
         if (st != EVO_OK) return st;
     }
-    if (ctx->plan_in_flight) {
-        // the pinned staging block is about to be overwritten: the previous upload must have been read
-        EVO_CUDA_TRY(ctx, cudaEventSynchronize(ctx->plan_consumed));
-        ctx->plan_in_flight = false;
+    if (ctx->cta_timing) {
+        st = evo::reserve_device(ctx, &ctx->d_cta_times, &ctx->d_cta_times_bytes, std::max<size_t>(max_ctas, 1) * 16);
+        if (st != EVO_OK) return st;
+        ctx->cta_times_n = static_cast<uint32_t>(plan.ranges.size());
     }
-    char* h = static_cast<char*>(ctx->h_plan);
-    auto put = [&](size_t o, const void* src, size_t bytes) { if (bytes) std::memcpy(h + o, src, bytes); };
-    put(o_sets, plan.sets.data(), plan.sets.size() * sizeof(SetRec));
-    put(o_members, plan.members.data(), plan.members.size() * sizeof(MemberRec));
-    put(o_ranges, plan.ranges.data(), plan.ranges.size() * sizeof(CtaRange));
-    put(o_goff, plan.group_off.data(), plan.group_off.size() * 4);
-    put(o_gdesc, plan.group_desc.data(), plan.group_desc.size() * 4);
-    EVO_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_plan, h, plan_bytes, cudaMemcpyHostToDevice, stream));
-    EVO_CUDA_TRY(ctx, cudaEventRecord(ctx->plan_consumed, stream));
-    ctx->plan_in_flight = true;
 
-    const char* d = static_cast<const char*>(ctx->d_plan);
-    const SetRec* d_sets = reinterpret_cast<const SetRec*>(d + o_sets);
-    const MemberRec* d_members = reinterpret_cast<const MemberRec*>(d + o_members);
-    const CtaRange* d_ranges = reinterpret_cast<const CtaRange*>(d + o_ranges);
-    Acc* d_parts = static_cast<Acc*>(ctx->d_partials);
-
-    const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
-    const cudaEvent_t ev_start = ctx->time_start, ev_stop = ctx->time_stop;
-    ctx->time_start = ctx->time_stop = nullptr;
-    if (ev_start) EVO_CUDA_TRY(ctx, cudaEventRecord(ev_start, stream));
-    uint32_t* d_status = evo::status_word(ctx);
-    const uint32_t* d_seeds = nullptr;
-    if (seed && n_desc > 0) {
-        seed_kernel<<<static_cast<unsigned>(n_desc), kThreads, 0, stream>>>(d_sets, d_members, static_cast<uint32_t*>(ctx->d_seeds));
-        ctx->launches += 1;
-        EVO_CUDA_TRY(ctx, cudaGetLastError());
-        d_seeds = static_cast<const uint32_t*>(ctx->d_seeds);
-    }
-    if (n_ctas > 0) {
-        if (!ctx->pass1_ready) {
-            EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(validate_pass1, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   static_cast<int>(kRingBytes)));
-            ctx->pass1_ready = true;
+    // ---- the plan goes up: as kernel arguments when it is small, else with a copy from pinned memory ----
+    if (L.bytes <= kPlanAsArgumentsLimit) {
+        std::vector<unsigned char> h(L.bytes);
+        pack_plan(plan, L, 0, h.data());
+        cudaError_t e = store_plan(h.data(), L.bytes, static_cast<unsigned char*>(ctx->d_plan), nullptr, ctx->pdl, stream, &ctx->launches);
+        if (e != cudaSuccess) return evo::fail_cuda(ctx, e, "plan_store launch");
+    } else {
+        st = evo::reserve_pinned(ctx, &ctx->h_plan, &ctx->h_plan_bytes, L.bytes);
+        if (st != EVO_OK) return st;
+        if (ctx->plan_in_flight) {
+            // the pinned staging block is about to be overwritten: the previous upload must have been read
+            EVO_CUDA_TRY(ctx, cudaEventSynchronize(ctx->plan_consumed));
+            ctx->plan_in_flight = false;
         }
-        validate_pass1<<<n_ctas, kBlock, kRingBytes, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol, d_status,
-                                                               d_seeds);
-        ctx->launches += 1;
-        EVO_CUDA_TRY(ctx, cudaGetLastError());
+        pack_plan(plan, L, 0, static_cast<unsigned char*>(ctx->h_plan));
+        EVO_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_plan, ctx->h_plan, L.bytes, cudaMemcpyHostToDevice, stream));
+        EVO_CUDA_TRY(ctx, cudaEventRecord(ctx->plan_consumed, stream));
+        ctx->plan_in_flight = true;
     }
-    if (ev_stop) EVO_CUDA_TRY(ctx, cudaEventRecord(ev_stop, stream));
-    const uint32_t n_members = static_cast<uint32_t>(n_desc);
-    if (n_members > 0) {
-        validate_pass2<<<(n_members + kWarps - 1) / kWarps, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts,
-                                                                                    n_members, results, d_status);
-        ctx->launches += 1;
-        EVO_CUDA_TRY(ctx, cudaGetLastError());
+
+    if (plan.ranges.size() > 0 && !ctx->pass1_ready) {
+        EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(validate_pass1, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>(kRingBytes)));
+        ctx->pass1_ready = true;
     }
-    if (group_pass) {
-        group_verdict<<<static_cast<unsigned>((n_group + 255) / 256), 256, 0, stream>>>(
-            reinterpret_cast<const uint32_t*>(d + o_goff), reinterpret_cast<const uint32_t*>(d + o_gdesc), results,
-            static_cast<uint32_t>(n_group), group_pass);
-        ctx->launches += 1;
-        EVO_CUDA_TRY(ctx, cudaGetLastError());
-    }
+    ChainArgs a{};
+    a.d_plan = static_cast<const unsigned char*>(ctx->d_plan);
+    a.L = L;
+    a.d_parts = static_cast<Acc*>(ctx->d_partials);
+    a.d_status = evo::status_word(ctx);
+    a.d_seeds = seed ? static_cast<uint32_t*>(ctx->d_seeds) : nullptr;
+    a.d_cta_times = ctx->cta_timing ? static_cast<unsigned long long*>(ctx->d_cta_times) : nullptr;
+    a.atol = atol; a.rtol = rtol;
+    a.results = results; a.group_pass = group_pass; a.n_group = n_group;
+    a.pdl = ctx->pdl;
+    a.ev_start = ev_start; a.ev_stop = ev_stop;
+    const cudaError_t e = launch_chain(plan, a, stream, &ctx->launches);
+    if (e != cudaSuccess) return evo::fail_cuda(ctx, e, "kernel launch");
     return EVO_OK;
 }
 
@@ -1043,13 +1208,8 @@ extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref
     if (st != EVO_OK) return static_fail(st, "evo_validate_static: %s", err.c_str());
 
     // Layout inside the scratch: the status word, the plan, then the partial records.
-    const size_t o_sets = kStaticStatusBytes;
-    const size_t o_members = align_up(o_sets + plan.sets.size() * sizeof(SetRec), 256);
-    const size_t o_ranges = align_up(o_members + plan.members.size() * sizeof(MemberRec), 256);
-    const size_t o_goff = align_up(o_ranges + plan.ranges.size() * sizeof(CtaRange), 256);
-    const size_t o_gdesc = align_up(o_goff + plan.group_off.size() * 4, 256);
-    const size_t plan_bytes = align_up(o_gdesc + plan.group_desc.size() * 4, 256);
-    const size_t o_parts = plan_bytes;
+    const PlanLayout L = layout_of(plan, kStaticStatusBytes);
+    const size_t o_parts = L.bytes;
     const size_t need = o_parts + static_cast<size_t>(plan.n_parts) * sizeof(Acc);
     if (need > kStaticScratchBytes)
         return static_fail(EVO_ERR_WORKSPACE,
@@ -1057,44 +1217,26 @@ extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref
                            "(%llu tensors in %zu sets); use evo_validate or split the call",
                            need, kStaticScratchBytes, (unsigned long long)n_desc, plan.sets.size());
 
-    // The plan goes up from ordinary host memory: the copy call returns once the runtime has
-    // taken the bytes, so the local buffer may go out of scope.
-    const size_t up_bytes = plan_bytes - kStaticStatusBytes;
-    std::vector<unsigned char> h(up_bytes ? up_bytes : 1);
-    auto put = [&](size_t o, const void* src, size_t bytes) { if (bytes) std::memcpy(h.data() + (o - kStaticStatusBytes), src, bytes); };
-    put(o_sets, plan.sets.data(), plan.sets.size() * sizeof(SetRec));
-    put(o_members, plan.members.data(), plan.members.size() * sizeof(MemberRec));
-    put(o_ranges, plan.ranges.data(), plan.ranges.size() * sizeof(CtaRange));
-    put(o_goff, plan.group_off.data(), plan.group_off.size() * 4);
-    put(o_gdesc, plan.group_desc.data(), plan.group_desc.size() * 4);
-    if (up_bytes) {
-        e = cudaMemcpyAsync(dev.scratch + kStaticStatusBytes, h.data(), up_bytes, cudaMemcpyHostToDevice, stream);
-        if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: plan upload: %s", cudaGetErrorString(e));
-    }
-    const unsigned char* d = dev.scratch;
-    const SetRec* d_sets = reinterpret_cast<const SetRec*>(d + o_sets);
-    const MemberRec* d_members = reinterpret_cast<const MemberRec*>(d + o_members);
-    const CtaRange* d_ranges = reinterpret_cast<const CtaRange*>(d + o_ranges);
-    Acc* d_parts = reinterpret_cast<Acc*>(dev.scratch + o_parts);
-    // Nothing in the plan or the partial records has to start at zero: pass 1 writes every
-    // record that pass 2 reads, so what an earlier call left behind is never looked at.  The
-    // status word is zero from the library image and is only ever raised (a wait that ran out
-    // in pass 1); it is deliberately not cleared, so that such a failure stays visible: every
-    // later call on this device then reports incomplete results.
+    // The plan travels as the arguments of small store kernels (one per 16 KiB), so the call never
+    // hands the runtime a pointer into this function's own memory and never makes the host wait
+    // for the stream.  The first store also clears the status word: each call reports its own
+    // waits only, and one that ran out long ago does not mark later results incomplete.
+    // Nothing else in the scratch has to start at zero: the first pass writes every partial record
+    // that the second pass reads.
+    std::vector<unsigned char> h(L.bytes - kStaticStatusBytes);
+    pack_plan(plan, L, kStaticStatusBytes, h.data());
     uint32_t* d_status = reinterpret_cast<uint32_t*>(dev.scratch);
-    const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
-    if (n_ctas > 0)
-        validate_pass1<<<n_ctas, kBlock, kRingBytes, stream>>>(d_sets, d_members, d_ranges, d_parts, atol, rtol, d_status,
-                                                               nullptr);
-    const uint32_t n_members = static_cast<uint32_t>(n_desc);
-    if (n_members > 0)
-        validate_pass2<<<(n_members + kWarps - 1) / kWarps, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts,
-                                                                                    n_members, results, d_status);
-    if (group_pass)
-        group_verdict<<<static_cast<unsigned>((n_group + 255) / 256), 256, 0, stream>>>(
-            reinterpret_cast<const uint32_t*>(d + o_goff), reinterpret_cast<const uint32_t*>(d + o_gdesc), results,
-            static_cast<uint32_t>(n_group), group_pass);
-    e = cudaGetLastError();
+    e = store_plan(h.data(), h.size(), dev.scratch + kStaticStatusBytes, d_status, false, stream, nullptr);
+    if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: plan store: %s", cudaGetErrorString(e));
+    ChainArgs a{};
+    a.d_plan = dev.scratch;
+    a.L = L;
+    a.d_parts = reinterpret_cast<Acc*>(dev.scratch + o_parts);
+    a.d_status = d_status;
+    a.atol = atol; a.rtol = rtol;
+    a.results = results; a.group_pass = group_pass; a.n_group = n_group;
+    a.pdl = false;
+    e = launch_chain(plan, a, stream, nullptr);
     if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: launch: %s", cudaGetErrorString(e));
     return EVO_OK;
 }

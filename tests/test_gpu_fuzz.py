@@ -96,3 +96,73 @@ def test_random_populations_with_a_few_tiles_per_cta(seed):
     each tensor's first tile."""
     rng = np.random.default_rng(7000 + seed)
     _run(_population(rng, 9000 + seed, sizes=[150001, 200000, 131072, 99999], n_refs=14))
+
+
+def _from_bits32(bits):
+    return torch.from_numpy(np.asarray(bits, dtype=np.uint32).view(np.float32).copy())
+
+
+def _adversarial(dtype, k, seed, filler_tensors=0):
+    """Full tiles whose quotients d/|r| live where the division-free filter of max d/|r| is most exposed:
+    subnormal references with differences of the same order (products and quotients under- and overflow),
+    a few normal elements mixed in so that the running maximum crosses the range where the approximate first-tile
+    quotients are trusted, and the largest quotient placed in the last lane of the first tile.
+    With `filler_tensors` the population has enough tiles for the seed pass to run."""
+    rng = np.random.default_rng(seed)
+    g = torch.Generator().manual_seed(seed)
+    tdt = TORCH[dtype]
+    n = 3 * 4096 + 777
+    if dtype == workloads.F32:
+        ref = _from_bits32(rng.integers(1, 1 << 14, n)) * torch.where(torch.rand(n, generator=g) < 0.5, -1.0, 1.0)   # 1e-45 .. 2e-41
+        tiny = lambda m: _from_bits32(rng.integers(0, 1 << 14, m))
+    else:
+        sub = torch.finfo(tdt).smallest_normal / (1 << (10 if dtype == workloads.F16 else 7))     # smallest subnormal
+        ref = (torch.from_numpy(rng.integers(1, 64, n)).float() * sub) * torch.where(torch.rand(n, generator=g) < 0.5, -1.0, 1.0)
+        tiny = lambda m: torch.from_numpy(rng.integers(0, 64, m)).float() * sub
+    ref = ref.to(tdt)
+    refs, tensors = [ref], []
+    for i in range(k):
+        c = ref.float() + tiny(n) * torch.where(torch.rand(n, generator=g) < 0.5, -1.0, 1.0)
+        if i % 3 == 1:                       # a few normal-range elements: quotients of order 1 among subnormal ones
+            idx = torch.randint(0, n, (5,), generator=g)
+            c[idx] = ref.float()[idx] * 3.0
+        if i % 3 == 2:                       # the largest quotient in the last element of the first tile
+            c[4095] = ref.float()[4095] * 40.0
+        if i % 4 == 3:                       # zeros in the candidate: d == |r|, quotient exactly 1
+            c[torch.randint(0, n, (50,), generator=g)] = 0.0
+        tensors.append(workloads.Tensor(c.to(tdt), 0, i % 7, dtype))
+    for j in range(filler_tensors):          # ordinary tensors that only add tiles
+        r = torch.randn(60000, generator=g).to(tdt)
+        refs.append(r)
+        tensors.append(workloads.Tensor((r.float() * (1 + 1e-3 * torch.randn(60000, generator=g))).to(tdt), len(refs) - 1, j % 7, dtype))
+    return workloads.Population("adversarial dtype %d k %d" % (dtype, k), refs, tensors, 7, 0.0, 1e-3,
+                                torch.ones(7, 1), torch.ones(1))
+
+
+@pytest.mark.parametrize("dtype", [workloads.F32, workloads.F16, workloads.BF16])
+@pytest.mark.parametrize("k", [1, 2, 33])
+def test_max_rel_filter_on_subnormal_references(dtype, k):
+    _run(_adversarial(dtype, k, 50 + k))
+
+
+@pytest.mark.parametrize("dtype", [workloads.F32, workloads.BF16])
+def test_max_rel_filter_on_subnormal_references_with_the_seed_pass(dtype):
+    """Same data inside a population large enough (at least as many tiles as CTAs, few tiles each) for the filter to be
+    seeded from every tensor's first tile."""
+    _run(_adversarial(dtype, 5, 91, filler_tensors=40))
+
+
+def test_max_rel_filter_when_the_tolerance_product_overflows():
+    """References of half the largest binary32 value with rtol large enough that rtol * |r| overflows to +Inf (every finite
+    difference is then within tolerance), candidates at all distances up to an overflowing difference."""
+    g = torch.Generator().manual_seed(5)
+    n = 3 * 4096 + 99
+    big = torch.finfo(torch.float32).max / 2
+    ref = torch.where(torch.rand(n, generator=g) < 0.5, -big, big)
+    cands = []
+    for i in range(3):
+        c = ref * (1 + (torch.rand(n, generator=g) - 0.5) * [1e-6, 1.0, 3.9][i])       # the last one overflows where signs flip
+        cands.append(c)
+    tensors = [workloads.Tensor(c, 0, i, workloads.F32) for i, c in enumerate(cands)]
+    pop = workloads.Population("tolerance overflow", [ref], tensors, 7, 0.0, 3.0, torch.ones(7, 1), torch.ones(1))
+    _run(pop)

@@ -136,11 +136,12 @@ def config3(device="cpu", n=1 << 20, k_per_dtype=64, special_rate=1e-6, boundary
                       _times(gid, 100, 3100, device), _times(1, 100, 3101, device)[0])
 
 
-def config4(device="cpu", n=1 << 28, k=16) -> Population:
+def config4(device="cpu", n=1 << 28, k=16, seed=4000) -> Population:
     """k fp32 candidates of n elements against one reference, noise 1e-6; exactly one
-    candidate is fully wrong (the reference rotated by n/2); atol = rtol = 1e-4."""
+    candidate is fully wrong (the reference rotated by n/2); atol = rtol = 1e-4.
+    Another `seed` gives other tensors of the same kind (disjoint samples for parallel baselines)."""
     atol, rtol = 1e-4, 1e-4
-    g = _gen(device, 4000)
+    g = _gen(device, seed)
     ref = torch.randn(n, generator=g, device=device, dtype=torch.float32)
     wrong = int(torch.randint(0, k, (1,), generator=_gen("cpu", 4099)).item())
     tensors = []
