@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include <string>
+#include <vector>
 
 #include "evo.h"
 
@@ -26,6 +27,13 @@ struct evo_ctx {
     cudaEvent_t plan_consumed = nullptr;                       // the last plan upload has been read
     bool plan_in_flight = false;
     cudaEvent_t time_start = nullptr, time_stop = nullptr;     // one-shot request of evo_set_timing_events
+    // What d_plan holds: the arguments of the evo_validate call whose plan was uploaded last (byte image), and what
+    // launching it takes.  A call with the same arguments skips planning and upload.
+    bool plan_key_valid = false;
+    std::vector<unsigned char> plan_key, plan_scratch_key;
+    size_t plan_layout[6] = {0, 0, 0, 0, 0, 0};
+    uint32_t plan_n_members = 0, plan_n_ctas = 0;
+    bool plan_seed = false;
     bool pdl = true;                                           // launch kernels so that they may overlap their predecessor's tail
     bool cta_timing = false;                                   // evo_debug_cta_timing: the first pass records per-CTA clocks
     void* d_cta_times = nullptr; size_t d_cta_times_bytes = 0; // two 64-bit %globaltimer readings per CTA

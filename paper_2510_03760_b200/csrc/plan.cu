@@ -48,7 +48,31 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
     if (n_desc > 0 && (!cand_ptrs || !descs)) return plan_fail(err, EVO_ERR_ARG, "cand_ptrs and descs must not be NULL");
     if (max_ctas == 0) return plan_fail(err, EVO_ERR_ARG, "max_ctas must be positive");
 
-    // ---- sets: tensors with the same (reference, n, dtype), at most kMaxK each ----
+    // ---- how many members a set may hold ----
+    // Up to kMaxK.  An item (set, tile) is the unit of the cut below, so a CTA's share is only even to
+    // within one item; when every CTA gets work but only a few items (a mid-sized population of many
+    // tensors per reference), smaller sets give more, lighter items at the price of reading the
+    // reference once more per extra set (from L2, mostly).
+    uint32_t cap = kMaxK;
+    {
+        std::unordered_map<Key, uint32_t, KeyHash> members_of;
+        for (uint64_t i = 0; i < n_desc; ++i) {
+            const evo_desc& d = descs[i];
+            const int dt = d.dtype == -1 ? dtype : d.dtype;
+            if (d.n == 0 || dt < 0 || dt > 31 || dtype_bytes(dt) == 0) continue;      // judged below
+            members_of[Key{d.ref ? d.ref : ref_ptr, d.n, dt}] += 1;
+        }
+        auto items_with = [&](uint32_t c) {
+            unsigned __int128 items = 0;
+            for (const auto& kv : members_of)
+                items += static_cast<unsigned __int128>((kv.first.n + kTileElems - 1) / kTileElems) * ((kv.second + c - 1) / c);
+            return items;
+        };
+        if (items_with(kMaxK) >= max_ctas)
+            while (cap > 4 && items_with(cap) < static_cast<unsigned __int128>(6) * max_ctas) cap /= 2;
+    }
+
+    // ---- sets: tensors with the same (reference, n, dtype), at most `cap` each ----
     std::unordered_map<Key, uint32_t, KeyHash> open;       // key -> set still accepting members
     std::vector<SetRec>& sets = plan->sets;
     sets.clear();
@@ -70,7 +94,7 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
         const Key key{d.n ? ref : nullptr, d.n, dt};
         auto it = open.find(key);
         uint32_t s;
-        if (it == open.end() || sets[it->second].k == kMaxK) {
+        if (it == open.end() || sets[it->second].k == cap) {
             s = static_cast<uint32_t>(sets.size());
             SetRec S{};
             S.ref = ref; S.n = d.n; S.k = 0; S.dtype = static_cast<uint32_t>(dt);

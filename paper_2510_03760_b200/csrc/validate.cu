@@ -49,9 +49,8 @@ namespace {
 using namespace evo;
 
 constexpr int kCtasPerSm = 2;
-constexpr int kStages = 12;                         // ring depth per CTA
-constexpr int kStageBytes = kTileElems * 2;         // 8 KiB: one 16-bit tile; an fp32 tile travels as two stages
-constexpr int kStageVecs = kStageBytes / (16 * kThreads);   // 16-byte vectors per consumer thread and stage (2)
+constexpr int kStages = 6;                          // ring depth per CTA
+constexpr int kStageBytes = kTileElems * 4;         // 16 KiB: one fp32 tile (a 16-bit tile uses half)
 constexpr size_t kRingBytes = static_cast<size_t>(kStages) * kStageBytes;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait, then give up
 constexpr uint64_t kSeedBelowTilesPerCta = 32;               // runs shorter than this get the seed pass
@@ -121,6 +120,11 @@ __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" 
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 __device__ __forceinline__ float rcp_approx(float x) {
     float y;
     asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -237,21 +241,17 @@ __device__ __forceinline__ void ring_release(Ring& g, int lane) {
     g.advance();
 }
 
-// One tile (kTileElems elements of one tensor) out of the ring into registers: it arrives as one
-// stage (16-bit types) or two consecutive stages (fp32); thread t's vector v is vector
-// (v mod kStageVecs) * kThreads + t of stage v / kStageVecs.  Each stage is handed back as soon
-// as the warp has its share.  False if a wait ran out.
+// One tile (kTileElems elements of one tensor) out of the ring into registers: thread t takes
+// vectors v * kThreads + t of the stage, which is handed back as soon as the warp has its share.
+// False if a wait ran out.
 template <int DT>
 __device__ __forceinline__ bool take_tile(Ring& g, uint4 (&v)[Elem<DT>::kVecs], int lane) {
     constexpr uint32_t kVecStride = kThreads * 16;
+    if (!ring_acquire(g)) return false;
+    const uint32_t a = g.data() + threadIdx.x * 16;
 #pragma unroll
-    for (int p = 0; p < Elem<DT>::kVecs / kStageVecs; ++p) {
-        if (!ring_acquire(g)) return false;
-        const uint32_t a = g.data() + threadIdx.x * 16;
-#pragma unroll
-        for (int q = 0; q < kStageVecs; ++q) v[p * kStageVecs + q] = lds128(a + q * kVecStride);
-        ring_release(g, lane);
-    }
+    for (int q = 0; q < Elem<DT>::kVecs; ++q) v[q] = lds128(a + q * kVecStride);
+    ring_release(g, lane);
     return true;
 }
 
@@ -260,23 +260,25 @@ __device__ __forceinline__ bool take_tile(Ring& g, uint4 (&v)[Elem<DT>::kVecs], 
 __device__ __noinline__ float div_rn(float a, float b) { return __fdiv_rn(a, b); }
 
 constexpr float kInf = __builtin_huge_valf();
-constexpr float kShrink = 0.99999904632568359375f;      // 1 - 2^-20
 
 // One full, 16-byte aligned tile: reference into registers once, then every member.
 //
 // Fast path per element, valid when c and r are finite and d does not overflow: d = |c - r|,
-// its maximum and its square; mismatches are counted only for a thread whose largest d exceeds
-// the smallest tolerance of its elements.  With atol, rtol >= 0 and finite data c == r implies
-// d = 0 <= tol, so the equality clause needs no test here.
-// The quotient d/|r| is not formed: `mlo` is slightly below the running maximum m of the
-// quotient, and d > RZ(mlo*|r|) holds whenever fl(d/|r|) > m could (rounding the product
-// toward zero keeps the test one-sided), so a miss never loses a maximum.  A thread whose
-// filter fired walks its 16 elements again in registers and divides only where r != 0 and
-// the filter still fires against its own, rising maximum.
+// its maximum and its square; mismatches are counted only in a group of elements (a 16-byte vector of a
+// 16-bit type, the thread's 16 elements of fp32) whose largest d exceeds the smallest tolerance of the
+// group.  With atol, rtol >= 0 and finite data c == r implies d = 0 <= tol, so the equality clause
+// needs no test here.
+// The quotient d/|r| is not formed.  With m the running maximum of the quotient (a binary32 value),
+// fl(d/|r|) > m implies d/|r| > m (rounding is monotone and m is representable), hence
+// d > m*|r| >= RZ(m*|r|): the test d > RZ(m*|r|) never misses a new maximum, and an element that only
+// ties the maximum does not pass it.  A thread whose filter fired walks its 16 elements again in
+// registers and divides only where r != 0 and the filter still fires against its own, rising maximum.
 template <int DT>
 __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, float atol, float rtol, Acc (*s_acc)[kWarps],
                                           uint32_t* s_mr, const void* const* s_cand, Ring& g, int warp, int lane) {
     using E = Elem<DT>;
+    constexpr int kGroups = E::kTolGroups;          // groups of elements with a smallest tolerance of their own
+    constexpr int kPerGroup = kEpt / kGroups;
     if (g.dead) return;
     float r[kEpt];
     {
@@ -287,13 +289,17 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
 #pragma unroll
             for (int e = 0; e < E::kPerVec; ++e) r[v * E::kPerVec + e] = E::at(rv[v], e);
     }
-    // The smallest tolerance among this thread's 16 reference elements: tol = atol + rtol*|r| does not decrease
-    // with |r| (each rounding is monotone), so it is the tolerance of the smallest |r|.  A member whose largest
-    // difference over these elements stays within it has no mismatch here, and none is counted element by element.
-    float armin = kInf;
+    // The smallest tolerance among a group's reference elements: tol = atol + rtol*|r| does not decrease with |r|
+    // (each rounding is monotone), so it is the tolerance of the smallest |r|.  A member whose largest difference
+    // over the group stays within it has no mismatch there, and none is counted element by element.
+    float tolmin[kGroups];
 #pragma unroll
-    for (int e = 0; e < kEpt; ++e) armin = fminf(armin, fabsf(r[e]));
-    const float tolmin = __fadd_rn(atol, __fmul_rn(rtol, armin));
+    for (int q = 0; q < kGroups; ++q) {
+        float armin = kInf;
+#pragma unroll
+        for (int e = 0; e < kPerGroup; ++e) armin = fminf(armin, fabsf(r[q * kPerGroup + e]));
+        tolmin[q] = __fadd_rn(atol, __fmul_rn(rtol, armin));
+    }
     const uint64_t vec0 = t * (kTileElems / E::kPerVec) + threadIdx.x;   // this thread's first vector of the tile
 #pragma unroll 1
     for (int k = 0; k < K; ++k) {
@@ -303,37 +309,48 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
         // Running maximum of d/|r| of this member, shared by the CTA's warps.  A stale (smaller)
         // value only makes the filter fire more often.
         const float m = __uint_as_float(*reinterpret_cast<volatile uint32_t*>(&s_mr[k]));
-        const float mlo = __fmul_rz(m, kShrink);
         uint32_t cnt = 0;
-        float ma = 0.f, sse = 0.f;
+        float sse = 0.f;
+        float mag[kGroups];
         bool trig = false;
 #pragma unroll
-        for (int v = 0; v < E::kVecs; ++v)
+        for (int q = 0; q < kGroups; ++q) {
+            mag[q] = 0.f;
 #pragma unroll
-            for (int e = 0; e < E::kPerVec; ++e) {
-                const int i = v * E::kPerVec + e;
-                const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
-                ma = fmaxf(ma, d);
-                sse = fmaf(d, d, sse);
-                trig |= d > __fmul_rz(mlo, fabsf(r[i]));
+            for (int e = 0; e < kPerGroup; e += 2) {
+                const int i = q * kPerGroup + e;
+                const float d0 = fabsf(__fsub_rn(E::at(cv[i / E::kPerVec], i % E::kPerVec), r[i]));
+                const float d1 = fabsf(__fsub_rn(E::at(cv[(i + 1) / E::kPerVec], (i + 1) % E::kPerVec), r[i + 1]));
+                mag[q] = max3(mag[q], d0, d1);
+                sse = fmaf(d0, d0, sse);
+                sse = fmaf(d1, d1, sse);
+                trig |= d0 > __fmul_rz(m, fabsf(r[i]));
+                trig |= d1 > __fmul_rz(m, fabsf(r[i + 1]));
             }
+        }
+        float ma = mag[0];
+#pragma unroll
+        for (int q = 1; q < kGroups; ++q) ma = fmaxf(ma, mag[q]);
         // The fast numbers do not stand if something was NaN/Inf or overflowed (the sum of
         // squares is then NaN/Inf) or if every d is so small that d^2 underflows in binary32.
         const bool redo = !(sse < kInf) || (ma < 9.094947017729282e-13f /* 2^-40 */ && ma > 0.f);
-        if (ma > tolmin && !redo) {
-            // some difference may exceed its tolerance: count, element by element
+        if (!redo) {
 #pragma unroll
-            for (int v = 0; v < E::kVecs; ++v)
+            for (int q = 0; q < kGroups; ++q) {
+                if (mag[q] > tolmin[q]) {
+                    // some difference of this group may exceed its tolerance: count, element by element
 #pragma unroll
-                for (int e = 0; e < E::kPerVec; ++e) {
-                    const int i = v * E::kPerVec + e;
-                    const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
-                    const float tol = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r[i])));
-                    cnt += (d > tol) ? 1u : 0u;
+                    for (int e = 0; e < kPerGroup; ++e) {
+                        const int i = q * kPerGroup + e;
+                        const float d = fabsf(__fsub_rn(E::at(cv[i / E::kPerVec], i % E::kPerVec), r[i]));
+                        const float tol = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r[i])));
+                        cnt += (d > tol) ? 1u : 0u;
+                    }
                 }
+            }
         }
         float mt = m;
-        float lo = mlo;
+        float lo = m;
         bool scan = trig && !redo;
         const unsigned full = 0xffffffffu;
         if (m == 0.f && __any_sync(full, scan)) {
@@ -371,7 +388,7 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
                     const float ar = fabsf(r[i]);
                     if (ar != 0.f && d > __fmul_rz(lo, ar)) {
                         const float q = div_rn(d, ar);
-                        if (q > mt) { mt = q; lo = __fmul_rz(mt, kShrink); }
+                        if (q > mt) { mt = q; lo = q; }
                     }
                 }
         }
@@ -421,23 +438,16 @@ __device__ __noinline__ void slow_tile(const SetRec& S, uint64_t t, float atol, 
     }
 }
 
-// The whole vectors of a ragged last tile: only the stages that hold some of its `valid_vecs`
-// vectors were copied (the producer counts the same way); vectors that do not exist read as zero.
+// The whole vectors of a ragged last tile (`valid_vecs` of them); vectors that do not exist read as zero.
 template <int DT>
 __device__ __forceinline__ bool take_tail(Ring& g, uint4 (&v)[Elem<DT>::kVecs], uint32_t valid_vecs, int lane) {
     constexpr uint32_t kVecStride = kThreads * 16;
+    if (!ring_acquire(g)) return false;
+    const uint32_t a = g.data() + threadIdx.x * 16;
 #pragma unroll
-    for (int p = 0; p < Elem<DT>::kVecs / kStageVecs; ++p) {
-#pragma unroll
-        for (int q = 0; q < kStageVecs; ++q) v[p * kStageVecs + q] = make_uint4(0u, 0u, 0u, 0u);
-        if (static_cast<uint32_t>(p) * kStageVecs * kThreads >= valid_vecs) continue;      // uniform for the CTA
-        if (!ring_acquire(g)) return false;
-        const uint32_t a = g.data() + threadIdx.x * 16;
-#pragma unroll
-        for (int q = 0; q < kStageVecs; ++q)
-            if ((p * kStageVecs + q) * kThreads + threadIdx.x < valid_vecs) v[p * kStageVecs + q] = lds128(a + q * kVecStride);
-        ring_release(g, lane);
-    }
+    for (int q = 0; q < Elem<DT>::kVecs; ++q)
+        v[q] = q * kThreads + threadIdx.x < valid_vecs ? lds128(a + q * kVecStride) : make_uint4(0u, 0u, 0u, 0u);
+    ring_release(g, lane);
     return true;
 }
 
@@ -587,25 +597,21 @@ __device__ __forceinline__ uint32_t producer_loop(const SetRec* __restrict__ set
         for (uint64_t t = t0; t < t1 && !g.dead; ++t) {
             const unsigned long long off = t * full_bytes;
             const uint32_t tile_bytes = t < sp.full_tiles ? full_bytes : sp.tail_vecs * 16u;
-            for (uint32_t j = 0; j <= S.k && !g.dead; ++j) {
+            for (uint32_t j = 0; j <= S.k; ++j) {
                 const unsigned long long base = __shfl_sync(full, mine, j == 0 ? 0 : static_cast<int>(j - 1));
                 const unsigned long long src = (j == 0 ? ref : base) + off;
-                // the tile in pieces of one stage each (one piece for 16-bit types, two for fp32, the last maybe short)
-                for (uint32_t done = 0; done < tile_bytes; done += kStageBytes) {
-                    const uint32_t piece = tile_bytes - done < static_cast<uint32_t>(kStageBytes) ? tile_bytes - done : kStageBytes;
-                    int ok = 1;
-                    if (lane == 0) {
-                        ok = mbar_wait(g.empty(), g.phase ^ 1u, g.abort_flag) ? 1 : 0;
-                        if (ok) {
-                            mbar_arrive_expect_tx(g.full(), piece);
-                            bulk_load(g.data(), reinterpret_cast<const void*>(src + done), piece, g.full(), pol);
-                        }
+                int ok = 1;
+                if (lane == 0) {
+                    ok = mbar_wait(g.empty(), g.phase ^ 1u, g.abort_flag) ? 1 : 0;
+                    if (ok) {
+                        mbar_arrive_expect_tx(g.full(), tile_bytes);
+                        bulk_load(g.data(), reinterpret_cast<const void*>(src), tile_bytes, g.full(), pol);
                     }
-                    ok = __shfl_sync(full, ok, 0);
-                    if (!ok) { g.dead = true; break; }
-                    g.advance();
-                    ++issued;
                 }
+                ok = __shfl_sync(full, ok, 0);
+                if (!ok) { g.dead = true; break; }
+                g.advance();
+                ++issued;
             }
         }
     }
@@ -926,14 +932,12 @@ struct ChainArgs {
     cudaEvent_t ev_start, ev_stop;    // optional: around the first pass
 };
 
-cudaError_t launch_chain(const Plan& plan, const ChainArgs& a, cudaStream_t stream, uint64_t* launches) {
+cudaError_t launch_chain(uint32_t n_members, uint32_t n_ctas, const ChainArgs& a, cudaStream_t stream, uint64_t* launches) {
     const SetRec* d_sets = reinterpret_cast<const SetRec*>(a.d_plan + a.L.o_sets);
     const MemberRec* d_members = reinterpret_cast<const MemberRec*>(a.d_plan + a.L.o_members);
     const CtaRange* d_ranges = reinterpret_cast<const CtaRange*>(a.d_plan + a.L.o_ranges);
     const uint32_t* d_goff = reinterpret_cast<const uint32_t*>(a.d_plan + a.L.o_goff);
     const uint32_t* d_gdesc = reinterpret_cast<const uint32_t*>(a.d_plan + a.L.o_gdesc);
-    const uint32_t n_members = static_cast<uint32_t>(plan.members.size());
-    const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
     cudaError_t e;
     auto count = [&]() { if (launches) *launches += 1; };
     if (a.d_seeds && n_members > 0) {
@@ -972,6 +976,23 @@ cudaError_t launch_chain(const Plan& plan, const ChainArgs& a, cudaStream_t stre
 
 constexpr size_t kPlanAsArgumentsLimit = 2 * kPlanChunkBytes;      // larger plans go up with a copy from pinned memory
 
+// Byte image of everything the plan depends on.
+void plan_key_of(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs, uint64_t n_desc, int dtype,
+                 bool want_groups, uint64_t n_group, uint32_t max_ctas, cudaStream_t stream, std::vector<unsigned char>* key) {
+    // (the stream is part of it: the upload is ordered on the stream of the call that made it)
+    struct Head { const void* ref; const void* stream; uint64_t n_desc, n_group; int32_t dtype; uint32_t max_ctas; uint32_t groups; uint32_t pad; } head;
+    std::memset(&head, 0, sizeof head);
+    head.ref = ref_ptr; head.stream = stream; head.n_desc = n_desc; head.n_group = n_group; head.dtype = dtype; head.max_ctas = max_ctas;
+    head.groups = want_groups ? 1u : 0u;
+    key->resize(sizeof head + n_desc * (sizeof(void*) + sizeof(evo_desc)));
+    unsigned char* p = key->data();
+    std::memcpy(p, &head, sizeof head);
+    if (n_desc) {
+        std::memcpy(p + sizeof head, cand_ptrs, n_desc * sizeof(void*));
+        std::memcpy(p + sizeof head + n_desc * sizeof(void*), descs, n_desc * sizeof(evo_desc));
+    }
+}
+
 int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs,
                     uint64_t n_desc, int dtype, float atol, float rtol, evo_result* results,
                     uint32_t* group_pass, uint64_t n_group, cudaStream_t stream, const char* who) {
@@ -979,56 +1000,81 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     const cudaEvent_t ev_start = ctx->time_start, ev_stop = ctx->time_stop;
     ctx->time_start = ctx->time_stop = nullptr;
     if (n_desc > 0 && !results) return evo::fail(ctx, EVO_ERR_ARG, "%s: results must not be NULL", who);
-    Plan plan;
-    std::string err;
+    if (!(atol >= 0.f) || !(rtol >= 0.f) || std::isinf(atol) || std::isinf(rtol))
+        return evo::fail(ctx, EVO_ERR_ARG, "%s: atol and rtol must be finite and >= 0", who);
+    if (n_desc > 0 && (!cand_ptrs || !descs)) return evo::fail(ctx, EVO_ERR_ARG, "%s: cand_ptrs and descs must not be NULL", who);
     const uint32_t max_ctas = static_cast<uint32_t>(ctx->sm_count) * kCtasPerSm;
-    int st = build_plan(cand_ptrs, ref_ptr, descs, n_desc, dtype, atol, rtol, group_pass != nullptr, n_group, max_ctas,
-                        &plan, &err);
-    if (st != EVO_OK) return evo::fail(ctx, st, "%s: %s", who, err.c_str());
 
     evo::DeviceGuard guard(ctx->device);
     if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
 
-    const PlanLayout L = layout_of(plan, 0);
-    st = evo::reserve_device(ctx, &ctx->d_plan, &ctx->d_plan_bytes, L.bytes + 256);
-    if (st != EVO_OK) return st;
-    st = evo::reserve_device(ctx, &ctx->d_partials, &ctx->d_partials_bytes, std::max<size_t>(plan.n_parts, 1) * sizeof(Acc));
-    if (st != EVO_OK) return st;
-    // Short runs (few tiles per CTA and member): seed the filter of max d/|r| first, see seed_kernel.
-    // (Not for populations with fewer tiles than CTAs: those are bound by launch latency, which a further
-    // kernel only adds to.)
-    const bool seed = plan.total_tiles >= max_ctas && plan.total_tiles / max_ctas < kSeedBelowTilesPerCta && n_desc > 0;
-    if (seed) {
-        st = evo::reserve_device(ctx, &ctx->d_seeds, &ctx->d_seeds_bytes, n_desc * sizeof(uint32_t));
+    // The same tensors as in the call before (an evaluation loop that reuses its buffers): the plan that is
+    // already in device memory stands, only the kernels are launched again.
+    std::vector<unsigned char>& key = ctx->plan_scratch_key;
+    plan_key_of(cand_ptrs, ref_ptr, descs, n_desc, dtype, group_pass != nullptr, n_group, max_ctas, stream, &key);
+    const bool hit = ctx->plan_key_valid && key.size() == ctx->plan_key.size() &&
+                     std::memcmp(key.data(), ctx->plan_key.data(), key.size()) == 0;
+    PlanLayout L;
+    uint32_t n_members, n_ctas;
+    bool seed;
+    if (hit) {
+        L = PlanLayout{ctx->plan_layout[0], ctx->plan_layout[1], ctx->plan_layout[2], ctx->plan_layout[3], ctx->plan_layout[4],
+                       ctx->plan_layout[5]};
+        n_members = ctx->plan_n_members; n_ctas = ctx->plan_n_ctas; seed = ctx->plan_seed;
+    } else {
+        Plan plan;
+        std::string err;
+        int st = build_plan(cand_ptrs, ref_ptr, descs, n_desc, dtype, atol, rtol, group_pass != nullptr, n_group, max_ctas,
+                            &plan, &err);
+        if (st != EVO_OK) return evo::fail(ctx, st, "%s: %s", who, err.c_str());
+        ctx->plan_key_valid = false;
+        L = layout_of(plan, 0);
+        n_members = static_cast<uint32_t>(plan.members.size());
+        n_ctas = static_cast<uint32_t>(plan.ranges.size());
+        st = evo::reserve_device(ctx, &ctx->d_plan, &ctx->d_plan_bytes, L.bytes + 256);
         if (st != EVO_OK) return st;
+        st = evo::reserve_device(ctx, &ctx->d_partials, &ctx->d_partials_bytes, std::max<size_t>(plan.n_parts, 1) * sizeof(Acc));
+        if (st != EVO_OK) return st;
+        // Short runs (few tiles per CTA and member): seed the filter of max d/|r| first, see seed_kernel.
+        // (Not for populations with fewer tiles than CTAs: those are bound by launch latency, which a further
+        // kernel only adds to.)
+        seed = plan.total_tiles >= max_ctas && plan.total_tiles / max_ctas < kSeedBelowTilesPerCta && n_desc > 0;
+        if (seed) {
+            st = evo::reserve_device(ctx, &ctx->d_seeds, &ctx->d_seeds_bytes, n_desc * sizeof(uint32_t));
+            if (st != EVO_OK) return st;
+        }
+        // ---- the plan goes up: as kernel arguments when it is small, else with a copy from pinned memory ----
+        if (L.bytes <= kPlanAsArgumentsLimit) {
+            std::vector<unsigned char> h(L.bytes);
+            pack_plan(plan, L, 0, h.data());
+            cudaError_t e = store_plan(h.data(), L.bytes, static_cast<unsigned char*>(ctx->d_plan), nullptr, ctx->pdl, stream, &ctx->launches);
+            if (e != cudaSuccess) return evo::fail_cuda(ctx, e, "plan_store launch");
+        } else {
+            st = evo::reserve_pinned(ctx, &ctx->h_plan, &ctx->h_plan_bytes, L.bytes);
+            if (st != EVO_OK) return st;
+            if (ctx->plan_in_flight) {
+                // the pinned staging block is about to be overwritten: the previous upload must have been read
+                EVO_CUDA_TRY(ctx, cudaEventSynchronize(ctx->plan_consumed));
+                ctx->plan_in_flight = false;
+            }
+            pack_plan(plan, L, 0, static_cast<unsigned char*>(ctx->h_plan));
+            EVO_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_plan, ctx->h_plan, L.bytes, cudaMemcpyHostToDevice, stream));
+            EVO_CUDA_TRY(ctx, cudaEventRecord(ctx->plan_consumed, stream));
+            ctx->plan_in_flight = true;
+        }
+        ctx->plan_key.swap(key);
+        ctx->plan_layout[0] = L.o_sets; ctx->plan_layout[1] = L.o_members; ctx->plan_layout[2] = L.o_ranges;
+        ctx->plan_layout[3] = L.o_goff; ctx->plan_layout[4] = L.o_gdesc; ctx->plan_layout[5] = L.bytes;
+        ctx->plan_n_members = n_members; ctx->plan_n_ctas = n_ctas; ctx->plan_seed = seed;
+        ctx->plan_key_valid = true;
     }
     if (ctx->cta_timing) {
-        st = evo::reserve_device(ctx, &ctx->d_cta_times, &ctx->d_cta_times_bytes, std::max<size_t>(max_ctas, 1) * 16);
+        const int st = evo::reserve_device(ctx, &ctx->d_cta_times, &ctx->d_cta_times_bytes, std::max<size_t>(max_ctas, 1) * 16);
         if (st != EVO_OK) return st;
-        ctx->cta_times_n = static_cast<uint32_t>(plan.ranges.size());
+        ctx->cta_times_n = n_ctas;
     }
 
-    // ---- the plan goes up: as kernel arguments when it is small, else with a copy from pinned memory ----
-    if (L.bytes <= kPlanAsArgumentsLimit) {
-        std::vector<unsigned char> h(L.bytes);
-        pack_plan(plan, L, 0, h.data());
-        cudaError_t e = store_plan(h.data(), L.bytes, static_cast<unsigned char*>(ctx->d_plan), nullptr, ctx->pdl, stream, &ctx->launches);
-        if (e != cudaSuccess) return evo::fail_cuda(ctx, e, "plan_store launch");
-    } else {
-        st = evo::reserve_pinned(ctx, &ctx->h_plan, &ctx->h_plan_bytes, L.bytes);
-        if (st != EVO_OK) return st;
-        if (ctx->plan_in_flight) {
-            // the pinned staging block is about to be overwritten: the previous upload must have been read
-            EVO_CUDA_TRY(ctx, cudaEventSynchronize(ctx->plan_consumed));
-            ctx->plan_in_flight = false;
-        }
-        pack_plan(plan, L, 0, static_cast<unsigned char*>(ctx->h_plan));
-        EVO_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_plan, ctx->h_plan, L.bytes, cudaMemcpyHostToDevice, stream));
-        EVO_CUDA_TRY(ctx, cudaEventRecord(ctx->plan_consumed, stream));
-        ctx->plan_in_flight = true;
-    }
-
-    if (plan.ranges.size() > 0 && !ctx->pass1_ready) {
+    if (n_ctas > 0 && !ctx->pass1_ready) {
         EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(validate_pass1, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                static_cast<int>(kRingBytes)));
         ctx->pass1_ready = true;
@@ -1044,7 +1090,7 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     a.results = results; a.group_pass = group_pass; a.n_group = n_group;
     a.pdl = ctx->pdl;
     a.ev_start = ev_start; a.ev_stop = ev_stop;
-    const cudaError_t e = launch_chain(plan, a, stream, &ctx->launches);
+    const cudaError_t e = launch_chain(n_members, n_ctas, a, stream, &ctx->launches);
     if (e != cudaSuccess) return evo::fail_cuda(ctx, e, "kernel launch");
     return EVO_OK;
 }
@@ -1236,7 +1282,7 @@ extern "C" int evo_validate_static(const void* const* cand_ptrs, const void* ref
     a.atol = atol; a.rtol = rtol;
     a.results = results; a.group_pass = group_pass; a.n_group = n_group;
     a.pdl = false;
-    e = launch_chain(plan, a, stream, nullptr);
+    e = launch_chain(static_cast<uint32_t>(plan.members.size()), static_cast<uint32_t>(plan.ranges.size()), a, stream, nullptr);
     if (e != cudaSuccess) return static_fail(EVO_ERR_CUDA, "evo_validate_static: launch: %s", cudaGetErrorString(e));
     return EVO_OK;
 }

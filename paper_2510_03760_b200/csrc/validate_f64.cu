@@ -291,6 +291,7 @@ extern "C" int evo_validate_f64(evo_ctx* ctx, const void* const* cand_ptrs, cons
     const size_t o_goff = align_up(o_ranges + plan.ranges.size() * sizeof(CtaRange), 256);
     const size_t o_gdesc = align_up(o_goff + plan.group_off.size() * 4, 256);
     const size_t plan_bytes = align_up(o_gdesc + plan.group_desc.size() * 4, 256) + 256;
+    ctx->plan_key_valid = false;          // the plan area is about to hold this call's plan
     st = evo::reserve_pinned(ctx, &ctx->h_plan, &ctx->h_plan_bytes, plan_bytes);
     if (st != EVO_OK) return st;
     st = evo::reserve_device(ctx, &ctx->d_plan, &ctx->d_plan_bytes, plan_bytes);

@@ -69,17 +69,36 @@ def tiles_of(n, dtype, tile_elems):
 
 
 def test_shared_reference_becomes_one_set_and_cut_is_balanced(lib):
-    n = 1 << 22
+    n = 1 << 25
     descs = np.zeros(16, DESC)
     descs["n"], descs["ref"], descs["dtype"] = n, 0x7000_0000_0000, F32
     cands = 0x1000_0000_0000 + np.arange(16, dtype=np.uint64) * (n * 4)
     st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
     assert st == 0 and summ["n_sets"] == 1 and set_k.tolist() == [16] and set(set_of.tolist()) == {0}
     tiles = tiles_of(n, F32, int(summ["tile_elems"]))
-    assert summ["total_tiles"] == tiles and summ["n_ctas"] == 444 and tiles > 444
+    assert summ["total_tiles"] == tiles and summ["n_ctas"] == 444 and tiles > 6 * 444
     w = coverage(summ, ranges, [tiles])
     assert max(w) - min(w) <= 1
     assert summ["n_parts"] == 444 * 16
+
+
+def test_few_items_per_cta_split_a_large_set_for_balance(lib):
+    """Every CTA gets work but fewer than six (set, tile) items: the members of one reference are spread over
+    smaller sets (never below four members), so that the shares of the CTAs come out more even."""
+    n = 1 << 22                                        # 1024 tiles for 444 CTAs
+    descs = np.zeros(16, DESC)
+    descs["n"], descs["ref"], descs["dtype"] = n, 0x7000_0000_0000, F32
+    cands = 0x1000_0000_0000 + np.arange(16, dtype=np.uint64) * (n * 4)
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
+    assert st == 0 and summ["n_sets"] == 4 and set_k.tolist() == [4, 4, 4, 4]
+    assert set_of.tolist() == [i // 4 for i in range(16)]
+    tiles = tiles_of(n, F32, int(summ["tile_elems"]))
+    w = coverage(summ, ranges, [tiles] * 4)
+    assert max(w) <= 1.12 * (sum(w) / len(w))          # shares within one item (5 tiles) of a mean of 46
+    # fewer tiles than CTAs: nothing to balance, one set
+    descs["n"] = 100 * 4096
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
+    assert st == 0 and summ["n_sets"] == 1 and summ["n_ctas"] == 100
 
 
 def test_more_members_than_a_set_holds(lib):
