@@ -264,10 +264,10 @@ constexpr float kInf = __builtin_huge_valf();
 // One full, 16-byte aligned tile: reference into registers once, then every member.
 //
 // Fast path per element, valid when c and r are finite and d does not overflow: d = |c - r|,
-// its maximum and its square; mismatches are counted only in a group of elements (a 16-byte vector of a
-// 16-bit type, the thread's 16 elements of fp32) whose largest d exceeds the smallest tolerance of the
-// group.  With atol, rtol >= 0 and finite data c == r implies d = 0 <= tol, so the equality clause
-// needs no test here.
+// its maximum and its square; mismatches are counted only in a group of elements (Elem::kTolGroups per
+// thread: one group of 16 measured fastest for every type) whose largest d exceeds the smallest
+// tolerance of the group.  With atol, rtol >= 0 and finite data c == r implies d = 0 <= tol, so the
+// equality clause needs no test here.
 // The quotient d/|r| is not formed.  With m the running maximum of the quotient (a binary32 value),
 // fl(d/|r|) > m implies d/|r| > m (rounding is monotone and m is representable), hence
 // d > m*|r| >= RZ(m*|r|): the test d > RZ(m*|r|) never misses a new maximum, and an element that only
