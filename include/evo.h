@@ -65,7 +65,7 @@ enum {
     EVO_ERR_TIMEOUT = -6     /* a bounded device-side wait gave up (reported through the context status word) */
 };
 
-/* Element types. EVO_U32 is accepted by evo_gen_inputs only; EVO_I32, EVO_I64 and EVO_U8 (also
+/* Element types. EVO_U32 is accepted by evo_gen_inputs and evo_validate_generated only; EVO_I32, EVO_I64 and EVO_U8 (also
  * the storage of bool) by evo_validate_exact only; EVO_F64 by evo_validate_f64 only. */
 enum { EVO_U32 = 0, EVO_F32 = 1, EVO_F16 = 2, EVO_BF16 = 3, EVO_F64 = 4, EVO_I32 = 5, EVO_I64 = 6, EVO_U8 = 7 };
 
@@ -274,6 +274,33 @@ EVO_API int evo_validate_exact(evo_ctx* ctx, const void* const* cand_ptrs /* hos
                                const void* ref_ptr /* device */, const evo_desc* descs /* host */, uint64_t n_desc, int dtype,
                                evo_result_exact* results /* device */, uint32_t* group_pass /* device, optional */,
                                uint64_t n_group, void* stream);
+
+/*
+ * evo_validate_generated - the equality check of evo_validate_exact against a reference that is
+ * not stored anywhere: a window of the random stream of evo_gen_inputs, regenerated inside the
+ * checking kernel.
+ * Paper: Section 4.3 (functional testing on random test cases; the stream of a test case is
+ * reproducible from its seed) and Section 3.1 Eq. 1.  Use: a buffer that must still hold, or must
+ * have been reproduced as, the raw words that evo_gen_inputs(seed, start, EVO_U32, n) writes - the
+ * inputs of a test case after the candidate ran (a kernel must not overwrite its inputs), or the
+ * output of a copying / reordering-free candidate - is checked without keeping a second copy and
+ * without reading one: per element the kernel spends ten Philox rounds per four words instead of
+ * four bytes of memory traffic.
+ * Tensor i holds counts[i] 32-bit elements and is compared with stream elements
+ * [start_i, start_i + counts[i]) of `seed`, start_i = offsets[i] (offsets NULL: `offset` for all);
+ * any start is accepted, multiples of 4 cost one Philox block per four elements, others two.
+ * dtype EVO_U32 compares the words as unsigned, EVO_I32 as two's-complement integers (only
+ * max_abs_diff differs).  Tensors with the same window are found and checked together.
+ * cand_ptrs : host array of n_desc device pointers (4-byte aligned; 16-byte aligned ones take the vector path).
+ * counts, offsets, groups : host arrays of n_desc entries (groups may be NULL without group_pass).
+ * results, group_pass, n_group : as evo_validate_exact.
+ * Errors: EVO_ERR_ARG, EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_WORKSPACE, EVO_ERR_CUDA.
+ */
+EVO_API int evo_validate_generated(evo_ctx* ctx, uint64_t seed, uint64_t offset, const uint64_t* offsets /* host, optional */,
+                                   const void* const* cand_ptrs /* host array of device ptrs */, const uint64_t* counts /* host */,
+                                   uint64_t n_desc, int dtype, const uint32_t* groups /* host, optional */,
+                                   evo_result_exact* results /* device */, uint32_t* group_pass /* device, optional */,
+                                   uint64_t n_group, void* stream);
 
 /*
  * evo_validate_f64 - the correctness constraint for binary64 outputs.

@@ -97,6 +97,8 @@ def load_library():
     L.evo_mismatch_sample.restype = i32
     L.evo_validate_exact.argtypes = [vp, vp, vp, vp, u64, i32, vp, vp, u64, vp]
     L.evo_validate_exact.restype = i32
+    L.evo_validate_generated.argtypes = [vp, u64, u64, vp, vp, vp, u64, i32, vp, vp, vp, u64, vp]
+    L.evo_validate_generated.restype = i32
     L.evo_validate_f64.argtypes = [vp, vp, vp, vp, u64, C.c_double, C.c_double, vp, vp, u64, vp]
     L.evo_validate_f64.restype = i32
     L.evo_plan_inspect.argtypes = [vp, vp, vp, u64, i32, u32, vp, vp, vp, vp]
@@ -319,6 +321,36 @@ def evo_validate_exact(cands, refs, groups=None, n_group=0, stream=None, ctx=Non
     group_pass = torch.empty(int(n_group), dtype=torch.int32, device=device) if groups is not None else None
     st = load_library().evo_validate_exact(
         ctx._h, C.c_void_p(ptrs.ctypes.data), None, C.c_void_p(descs.ctypes.data), n, EVO_I32, _dev_ptr(results),
+        _dev_ptr(group_pass) if groups is not None else None, int(n_group) if groups is not None else 0,
+        _stream_ptr(stream, device))
+    ctx.check(st)
+    return results, group_pass
+
+
+def evo_validate_generated(seed, cands, offsets=0, dtype=EVO_U32, groups=None, n_group=0, stream=None, ctx=None):
+    """int32 / uint32-storage CUDA tensors checked for equality against windows of the random stream of `seed`,
+    regenerated in the kernel: tensor i against stream elements [offsets[i], offsets[i] + numel) (`offsets` may be one
+    number for all).  dtype EVO_U32 or EVO_I32 says how the words compare.  Returns (results as evo_validate_exact,
+    group_pass or None)."""
+    n = len(cands)
+    device = cands[0].device if n else torch.device("cuda", torch.cuda.current_device())
+    ctx = ctx or default_context(device.index)
+    for i, c in enumerate(cands):
+        if not c.is_cuda or not c.is_contiguous() or c.element_size() != 4:
+            raise ValueError("tensor %d must be a contiguous CUDA tensor of 32-bit elements" % i)
+    ptrs = np.array([c.data_ptr() for c in cands], dtype=np.uint64)
+    counts = np.array([c.numel() for c in cands], dtype=np.uint64)
+    one = isinstance(offsets, int)
+    offs = None if one else np.ascontiguousarray(offsets, dtype=np.uint64)
+    if offs is not None and offs.size != n:
+        raise ValueError("need one stream offset per tensor, or a single number")
+    grp = np.ascontiguousarray(groups, dtype=np.uint32) if groups is not None else None
+    results = torch.empty((n, EXACT_DTYPE.itemsize), dtype=torch.uint8, device=device)
+    group_pass = torch.empty(int(n_group), dtype=torch.int32, device=device) if groups is not None else None
+    st = load_library().evo_validate_generated(
+        ctx._h, int(seed), int(offsets) if one else 0, C.c_void_p(offs.ctypes.data) if offs is not None else None,
+        C.c_void_p(ptrs.ctypes.data), C.c_void_p(counts.ctypes.data), n, int(dtype),
+        C.c_void_p(grp.ctypes.data) if grp is not None else None, _dev_ptr(results),
         _dev_ptr(group_pass) if groups is not None else None, int(n_group) if groups is not None else 0,
         _stream_ptr(stream, device))
     ctx.check(st)

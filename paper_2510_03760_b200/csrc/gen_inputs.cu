@@ -10,41 +10,11 @@
 #include <cuda_fp16.h>
 
 #include "evo_internal.h"
+#include "philox.cuh"
 
 namespace {
 
-constexpr uint32_t kPhiloxM0 = 0xD2511F53u;
-constexpr uint32_t kPhiloxM1 = 0xCD9E8D57u;
-constexpr uint32_t kPhiloxW0 = 0x9E3779B9u;
-constexpr uint32_t kPhiloxW1 = 0xBB67AE85u;
-
-// The ten round keys (key bumped by the Weyl constants before every round but the first) depend on the seed
-// only: the host works them out once and passes them as a kernel argument, so a round reads them as constant
-// operands instead of spending two additions.
-struct RoundKeys { uint32_t k0[10], k1[10]; };
-
-inline RoundKeys round_keys(uint64_t seed) {
-    RoundKeys rk;
-    uint32_t k0 = static_cast<uint32_t>(seed), k1 = static_cast<uint32_t>(seed >> 32);
-    for (int round = 0; round < 10; ++round) {
-        rk.k0[round] = k0; rk.k1[round] = k1;
-        k0 += kPhiloxW0; k1 += kPhiloxW1;
-    }
-    return rk;
-}
-
-__device__ __forceinline__ uint4 philox4x32_10(uint64_t block, const RoundKeys& rk) {
-    uint32_t c0 = static_cast<uint32_t>(block), c1 = static_cast<uint32_t>(block >> 32), c2 = 0u, c3 = 0u;
-#pragma unroll
-    for (int round = 0; round < 10; ++round) {
-        const uint32_t hi0 = __umulhi(kPhiloxM0, c0), lo0 = kPhiloxM0 * c0;
-        const uint32_t hi1 = __umulhi(kPhiloxM1, c2), lo1 = kPhiloxM1 * c2;
-        const uint32_t n0 = hi1 ^ c1 ^ rk.k0[round];
-        const uint32_t n2 = hi0 ^ c3 ^ rk.k1[round];
-        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
-    }
-    return make_uint4(c0, c1, c2, c3);
-}
+using namespace evo;
 
 // (xa, xb) -> (rho cos, rho sin).  u1 and 2*u2 are exact in binary32; the angle is handed
 // to sincospif as a multiple of pi so that no rounded 2*pi enters and the zeros at the

@@ -26,6 +26,11 @@ struct KeyHash {
     }
 };
 
+// Cost of one (set, tile) item: the tiles it moves (the reference and every member).  Other weightings were
+// measured on a ragged, mixed-type population and lost: 16-bit tiles lighter or heavier than fp32 ones, a
+// fixed cost per set.
+inline uint64_t item_weight(const SetRec& S) { return static_cast<uint64_t>(S.k) + 1; }
+
 int plan_fail(std::string* err, int status, const char* fmt, ...) {
     char buf[256];
     va_list ap;
@@ -130,7 +135,7 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
     for (uint32_t s = 0; s < n_sets; ++s) {
         tiles[s] = (sets[s].n + kTileElems - 1) / kTileElems;
         plan->total_tiles += tiles[s];
-        prefix[s + 1] = prefix[s] + static_cast<unsigned __int128>(tiles[s]) * (sets[s].k + 1);
+        prefix[s + 1] = prefix[s] + static_cast<unsigned __int128>(tiles[s]) * item_weight(sets[s]);
     }
     const unsigned __int128 total_cost = prefix[n_sets];
     const uint32_t n_ctas = static_cast<uint32_t>(std::min<uint64_t>(max_ctas, plan->total_tiles));
@@ -144,7 +149,7 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
             const unsigned __int128 pos = total_cost * b / n_ctas;
             while (s < n_sets && prefix[s + 1] <= pos) ++s;
             if (s == n_sets) cut[b] = {n_sets, 0};
-            else cut[b] = {s, static_cast<uint64_t>((pos - prefix[s]) / (sets[s].k + 1))};
+            else cut[b] = {s, static_cast<uint64_t>((pos - prefix[s]) / item_weight(sets[s]))};
         }
         for (uint32_t b = 0; b < n_ctas; ++b) {
             CtaRange R{};

@@ -58,7 +58,7 @@ struct CtaRange {            // items [(s_begin, t_begin), (s_end, t_end)) with 
 // Bytes per element of every type a plan can hold (0: not a type).
 inline uint32_t dtype_bytes(int dt) {
     switch (dt) {
-        case EVO_F32: case EVO_I32: return 4;
+        case EVO_F32: case EVO_I32: case EVO_U32: return 4;
         case EVO_F16: case EVO_BF16: return 2;
         case EVO_I64: case EVO_F64: return 8;
         case EVO_U8: return 1;
@@ -67,6 +67,7 @@ inline uint32_t dtype_bytes(int dt) {
 }
 constexpr uint32_t kFloatTypes = (1u << EVO_F32) | (1u << EVO_F16) | (1u << EVO_BF16);
 constexpr uint32_t kIntTypes = (1u << EVO_I32) | (1u << EVO_I64) | (1u << EVO_U8);
+constexpr uint32_t kWordTypes = (1u << EVO_I32) | (1u << EVO_U32);      // what a regenerated stream can be compared as
 
 struct Plan {
     std::vector<SetRec> sets;

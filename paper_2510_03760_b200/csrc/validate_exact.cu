@@ -14,7 +14,11 @@
 #include <cstring>
 #include <string>
 
+#include <unordered_map>
+#include <vector>
+
 #include "evo_internal.h"
+#include "philox.cuh"
 #include "plan.h"
 
 namespace {
@@ -225,6 +229,125 @@ exact_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ membe
     }
 }
 
+// ---- the reference regenerated in the kernel (evo_validate_generated) ----------------------
+// The reference of a set is a window of a Philox stream: SetRec::ref holds the stream position of
+// its first element instead of an address.  A thread produces the four words of a 16-byte vector
+// with one Philox block (two when the window does not start on a block boundary), so the reference
+// costs arithmetic and no memory traffic; the candidates stream through registers as above.
+template <bool SIGNED>
+__device__ __forceinline__ void word_pair(uint32_t c, uint32_t r, uint32_t& cnt, uint32_t& md) {
+    const bool gt = SIGNED ? static_cast<int32_t>(c) > static_cast<int32_t>(r) : c > r;
+    const uint32_t d = gt ? c - r : r - c;            // |c - r| of two 32-bit values fits 32 unsigned bits
+    cnt += d != 0 ? 1u : 0u;
+    md = max(md, d);
+}
+
+// Words [pos, pos + 4) of the stream, pos any value.
+__device__ __forceinline__ uint4 stream_vector(uint64_t pos, const RoundKeys& rk) {
+    const uint4 a = philox4x32_10(pos >> 2, rk);
+    const uint32_t lead = static_cast<uint32_t>(pos) & 3u;
+    if (lead == 0) return a;
+    const uint4 b = philox4x32_10((pos >> 2) + 1, rk);
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint4 v;
+    v.x = lead == 1 ? w[1] : lead == 2 ? w[2] : w[3];
+    v.y = lead == 1 ? w[2] : lead == 2 ? w[3] : w[4];
+    v.z = lead == 1 ? w[3] : lead == 2 ? w[4] : w[5];
+    v.w = lead == 1 ? w[4] : lead == 2 ? w[5] : w[6];
+    return v;
+}
+
+__device__ __forceinline__ uint32_t stream_word(uint64_t pos, const RoundKeys& rk) {
+    const uint4 a = philox4x32_10(pos >> 2, rk);
+    const uint32_t lane = static_cast<uint32_t>(pos) & 3u;
+    return lane == 0 ? a.x : lane == 1 ? a.y : lane == 2 ? a.z : a.w;
+}
+
+template <bool SIGNED>
+__device__ __forceinline__ void run_set_generated(const RoundKeys& rk, const SetRec& S, uint64_t t0, uint64_t t1,
+                                                  AccExact (*s_acc)[kWarps], const void* const* s_cand, int warp, int lane) {
+    constexpr int kVecs = kEpt / 4;                       // 16-byte vectors per thread per tile
+    constexpr int kTileVecs = kTileElems / 4;
+    const uint64_t first = reinterpret_cast<uint64_t>(S.ref);       // stream position of element 0
+    const uint64_t full_tiles = S.vec_ok ? S.n / kTileElems : 0;
+    for (uint64_t t = t0; t < t1; ++t) {
+        if (t < full_tiles) {
+            const uint64_t base = t * kTileVecs + threadIdx.x;
+            // the first member's loads are on their way while the reference is generated
+            uint4 c[kVecs];
+            {
+                const uint4* cp = static_cast<const uint4*>(s_cand[0]) + base;
+#pragma unroll
+                for (int v = 0; v < kVecs; ++v) c[v] = load_stream(cp + v * kThreads);
+            }
+            uint4 r[kVecs];
+#pragma unroll
+            for (int v = 0; v < kVecs; ++v) r[v] = stream_vector(first + 4 * (base + static_cast<uint64_t>(v) * kThreads), rk);
+#pragma unroll 1
+            for (uint32_t k = 0; k < S.k; ++k) {
+                if (k > 0) {
+                    const uint4* cp = static_cast<const uint4*>(s_cand[k]) + base;
+#pragma unroll
+                    for (int v = 0; v < kVecs; ++v) c[v] = load_stream(cp + v * kThreads);
+                }
+                uint32_t cnt = 0, md = 0;
+#pragma unroll
+                for (int v = 0; v < kVecs; ++v) {
+                    word_pair<SIGNED>(c[v].x, r[v].x, cnt, md); word_pair<SIGNED>(c[v].y, r[v].y, cnt, md);
+                    word_pair<SIGNED>(c[v].z, r[v].z, cnt, md); word_pair<SIGNED>(c[v].w, r[v].w, cnt, md);
+                }
+                commit(cnt, md, &s_acc[k][warp], lane);
+            }
+        } else {
+            // ragged last tile, or candidates that are not 16-byte aligned: element by element
+            const uint64_t e0 = t * kTileElems;
+            const uint64_t e1 = min(S.n, e0 + kTileElems);
+            for (uint64_t e = e0 + threadIdx.x; e < e0 + kTileElems; e += kThreads) {      // uniform trip count: commit is collective
+                const bool in = e < e1;
+                const uint32_t r = in ? stream_word(first + e, rk) : 0u;
+                for (uint32_t k = 0; k < S.k; ++k) {
+                    uint32_t cnt = 0, md = 0;
+                    if (in) word_pair<SIGNED>(static_cast<const uint32_t*>(s_cand[k])[e], r, cnt, md);
+                    commit(cnt, md, &s_acc[k][warp], lane);
+                }
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, kCtasPerSmExact)
+generated_pass1(const __grid_constant__ RoundKeys rk, const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
+                const CtaRange* __restrict__ ranges, AccExact* __restrict__ partials) {
+    __shared__ AccExact s_acc[kMaxK][kWarps];
+    __shared__ const void* s_cand[kMaxK];
+    const CtaRange rg = ranges[blockIdx.x];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (uint32_t s = rg.s_begin; s <= rg.s_end; ++s) {
+        const SetRec S = sets[s];
+        const uint64_t tiles = (S.n + kTileElems - 1) / kTileElems;
+        const uint64_t t0 = (s == rg.s_begin) ? rg.t_begin : 0;
+        const uint64_t t1 = (s == rg.s_end) ? rg.t_end : tiles;
+        if (t0 >= t1) continue;
+        for (uint32_t i = threadIdx.x; i < S.k * kWarps; i += kThreads) s_acc[i / kWarps][i % kWarps] = AccExact{0ull, 0ull};
+        if (threadIdx.x < S.k) s_cand[threadIdx.x] = members[S.member_off + threadIdx.x].cand;
+        __syncthreads();
+        if (S.dtype == EVO_I32) run_set_generated<true>(rk, S, t0, t1, s_acc, s_cand, warp, lane);
+        else run_set_generated<false>(rk, S, t0, t1, s_acc, s_cand, warp, lane);
+        __syncthreads();
+        if (threadIdx.x < S.k) {
+            AccExact a = s_acc[threadIdx.x][0];
+#pragma unroll
+            for (int w = 1; w < kWarps; ++w) {
+                const AccExact b = s_acc[threadIdx.x][w];
+                a.mism += b.mism;
+                a.maxdiff = b.maxdiff > a.maxdiff ? b.maxdiff : a.maxdiff;
+            }
+            partials[rg.part_base + (S.member_off - rg.first_member) + threadIdx.x] = a;
+        }
+        __syncthreads();
+    }
+}
+
 // One warp per tensor: fold the partial records of the CTAs [cta_first, cta_last] of its set.
 __global__ void __launch_bounds__(kThreads)
 exact_pass2(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members, const CtaRange* __restrict__ ranges,
@@ -268,25 +391,15 @@ __global__ void exact_verdict(const uint32_t* __restrict__ offsets, const uint32
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-}  // namespace
+// Device addresses of an uploaded plan.
+struct DevicePlan {
+    const SetRec* sets; const MemberRec* members; const CtaRange* ranges; const uint32_t* goff; const uint32_t* gdesc;
+    AccExact* parts;
+};
 
-extern "C" int evo_validate_exact(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs,
-                                  uint64_t n_desc, int dtype, evo_result_exact* results, uint32_t* group_pass,
-                                  uint64_t n_group, void* stream_) {
-    if (!ctx) return EVO_ERR_ARG;
-    const char* who = "evo_validate_exact";
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    if (n_desc > 0 && !results) return evo::fail(ctx, EVO_ERR_ARG, "%s: results must not be NULL", who);
-    Plan plan;
-    std::string err;
-    const uint32_t max_ctas = static_cast<uint32_t>(ctx->sm_count) * kCtasPerSmExact;
-    int st = build_plan(cand_ptrs, ref_ptr, descs, n_desc, dtype, 0.f, 0.f, group_pass != nullptr, n_group, max_ctas, &plan,
-                        &err, kIntTypes);
-    if (st != EVO_OK) return evo::fail(ctx, st, "%s: %s", who, err.c_str());
-    evo::DeviceGuard guard(ctx->device);
-    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
-
-    // pack and upload the plan (same staging as evo_validate: one pinned block, one copy)
+// Packs the plan into the context's pinned block, copies it to the device on `stream` and sizes the
+// partial records (one pinned block, one copy, as evo_validate does for large plans).
+int upload_plan(evo_ctx* ctx, const Plan& plan, cudaStream_t stream, DevicePlan* out) {
     const size_t o_sets = 0;
     const size_t o_members = align_up(o_sets + plan.sets.size() * sizeof(SetRec), 256);
     const size_t o_ranges = align_up(o_members + plan.members.size() * sizeof(MemberRec), 256);
@@ -294,7 +407,7 @@ extern "C" int evo_validate_exact(evo_ctx* ctx, const void* const* cand_ptrs, co
     const size_t o_gdesc = align_up(o_goff + plan.group_off.size() * 4, 256);
     const size_t plan_bytes = align_up(o_gdesc + plan.group_desc.size() * 4, 256) + 256;
     ctx->plan_key_valid = false;          // the plan area is about to hold this call's plan
-    st = evo::reserve_pinned(ctx, &ctx->h_plan, &ctx->h_plan_bytes, plan_bytes);
+    int st = evo::reserve_pinned(ctx, &ctx->h_plan, &ctx->h_plan_bytes, plan_bytes);
     if (st != EVO_OK) return st;
     st = evo::reserve_device(ctx, &ctx->d_plan, &ctx->d_plan_bytes, plan_bytes);
     if (st != EVO_OK) return st;
@@ -314,31 +427,114 @@ extern "C" int evo_validate_exact(evo_ctx* ctx, const void* const* cand_ptrs, co
     EVO_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_plan, h, plan_bytes, cudaMemcpyHostToDevice, stream));
     EVO_CUDA_TRY(ctx, cudaEventRecord(ctx->plan_consumed, stream));
     ctx->plan_in_flight = true;
-
     const char* d = static_cast<const char*>(ctx->d_plan);
-    const SetRec* d_sets = reinterpret_cast<const SetRec*>(d + o_sets);
-    const MemberRec* d_members = reinterpret_cast<const MemberRec*>(d + o_members);
-    const CtaRange* d_ranges = reinterpret_cast<const CtaRange*>(d + o_ranges);
-    AccExact* d_parts = static_cast<AccExact*>(ctx->d_partials);          // 16-byte records in a block sized for 40-byte ones
-    const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
-    if (n_ctas > 0) {
-        exact_pass1<<<n_ctas, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts);
-        ctx->launches += 1;
-        EVO_CUDA_TRY(ctx, cudaGetLastError());
-    }
+    out->sets = reinterpret_cast<const SetRec*>(d + o_sets);
+    out->members = reinterpret_cast<const MemberRec*>(d + o_members);
+    out->ranges = reinterpret_cast<const CtaRange*>(d + o_ranges);
+    out->goff = reinterpret_cast<const uint32_t*>(d + o_goff);
+    out->gdesc = reinterpret_cast<const uint32_t*>(d + o_gdesc);
+    out->parts = static_cast<AccExact*>(ctx->d_partials);          // 16-byte records in a block sized for 40-byte ones
+    return EVO_OK;
+}
+
+// Second pass and verdicts, the same after either first pass.
+int finish_exact(evo_ctx* ctx, const DevicePlan& d, uint64_t n_desc, evo_result_exact* results, uint32_t* group_pass,
+                 uint64_t n_group, cudaStream_t stream) {
     const uint32_t n_members = static_cast<uint32_t>(n_desc);
     if (n_members > 0) {
-        exact_pass2<<<(n_members + kWarps - 1) / kWarps, kThreads, 0, stream>>>(d_sets, d_members, d_ranges, d_parts, n_members,
+        exact_pass2<<<(n_members + kWarps - 1) / kWarps, kThreads, 0, stream>>>(d.sets, d.members, d.ranges, d.parts, n_members,
                                                                                  results);
         ctx->launches += 1;
         EVO_CUDA_TRY(ctx, cudaGetLastError());
     }
     if (group_pass) {
-        exact_verdict<<<static_cast<unsigned>((n_group + 255) / 256), 256, 0, stream>>>(
-            reinterpret_cast<const uint32_t*>(d + o_goff), reinterpret_cast<const uint32_t*>(d + o_gdesc), results,
-            static_cast<uint32_t>(n_group), group_pass);
+        exact_verdict<<<static_cast<unsigned>((n_group + 255) / 256), 256, 0, stream>>>(d.goff, d.gdesc, results,
+                                                                                        static_cast<uint32_t>(n_group), group_pass);
         ctx->launches += 1;
         EVO_CUDA_TRY(ctx, cudaGetLastError());
     }
     return EVO_OK;
+}
+
+}  // namespace
+
+extern "C" int evo_validate_exact(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_ptr, const evo_desc* descs,
+                                  uint64_t n_desc, int dtype, evo_result_exact* results, uint32_t* group_pass,
+                                  uint64_t n_group, void* stream_) {
+    if (!ctx) return EVO_ERR_ARG;
+    const char* who = "evo_validate_exact";
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (n_desc > 0 && !results) return evo::fail(ctx, EVO_ERR_ARG, "%s: results must not be NULL", who);
+    Plan plan;
+    std::string err;
+    const uint32_t max_ctas = static_cast<uint32_t>(ctx->sm_count) * kCtasPerSmExact;
+    int st = build_plan(cand_ptrs, ref_ptr, descs, n_desc, dtype, 0.f, 0.f, group_pass != nullptr, n_group, max_ctas, &plan,
+                        &err, kIntTypes);
+    if (st != EVO_OK) return evo::fail(ctx, st, "%s: %s", who, err.c_str());
+    evo::DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
+    DevicePlan d;
+    st = upload_plan(ctx, plan, stream, &d);
+    if (st != EVO_OK) return st;
+    const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
+    if (n_ctas > 0) {
+        exact_pass1<<<n_ctas, kThreads, 0, stream>>>(d.sets, d.members, d.ranges, d.parts);
+        ctx->launches += 1;
+        EVO_CUDA_TRY(ctx, cudaGetLastError());
+    }
+    return finish_exact(ctx, d, n_desc, results, group_pass, n_group, stream);
+}
+
+extern "C" int evo_validate_generated(evo_ctx* ctx, uint64_t seed, uint64_t offset, const uint64_t* offsets,
+                                      const void* const* cand_ptrs, const uint64_t* counts, uint64_t n_desc, int dtype,
+                                      const uint32_t* groups, evo_result_exact* results, uint32_t* group_pass,
+                                      uint64_t n_group, void* stream_) {
+    if (!ctx) return EVO_ERR_ARG;
+    const char* who = "evo_validate_generated";
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (dtype != EVO_I32 && dtype != EVO_U32) return evo::fail(ctx, EVO_ERR_DTYPE, "%s: dtype %d (EVO_I32 or EVO_U32)", who, dtype);
+    if (n_desc > 0 && (!results || !counts || !cand_ptrs))
+        return evo::fail(ctx, EVO_ERR_ARG, "%s: cand_ptrs, counts and results must not be NULL", who);
+    if (group_pass && n_desc > 0 && !groups) return evo::fail(ctx, EVO_ERR_ARG, "%s: group_pass without groups", who);
+    // Descriptors for the planner: tensors with the same window of the stream form a set, exactly as tensors
+    // with the same reference do.  The planner keys sets by the reference's address, so every distinct window
+    // start gets a stand-in address (16-byte aligned, never dereferenced), replaced by the stream position below.
+    std::vector<evo_desc> descs(n_desc);
+    std::unordered_map<uint64_t, uintptr_t> token_of;
+    std::vector<uint64_t> start_of_token;
+    for (uint64_t i = 0; i < n_desc; ++i) {
+        const uint64_t start = offsets ? offsets[i] : offset;
+        if (counts[i] > (1ull << 60)) return evo::fail(ctx, EVO_ERR_ARG, "%s: tensor %llu is too large", who, (unsigned long long)i);
+        auto it = token_of.find(start);
+        if (it == token_of.end()) {
+            start_of_token.push_back(start);
+            it = token_of.emplace(start, static_cast<uintptr_t>(16 * start_of_token.size())).first;
+        }
+        descs[i].n = counts[i];
+        descs[i].ref = reinterpret_cast<const void*>(it->second);
+        descs[i].dtype = dtype;
+        descs[i].group = groups ? groups[i] : 0u;
+    }
+    Plan plan;
+    std::string err;
+    const uint32_t max_ctas = static_cast<uint32_t>(ctx->sm_count) * kCtasPerSmExact;
+    int st = build_plan(cand_ptrs, nullptr, descs.data(), n_desc, dtype, 0.f, 0.f, group_pass != nullptr, n_group, max_ctas,
+                        &plan, &err, kWordTypes);
+    if (st != EVO_OK) return evo::fail(ctx, st, "%s: %s", who, err.c_str());
+    for (SetRec& S : plan.sets) {
+        const uintptr_t token = reinterpret_cast<uintptr_t>(S.ref);
+        S.ref = reinterpret_cast<const void*>(static_cast<uintptr_t>(token ? start_of_token[token / 16 - 1] : 0));
+    }
+    evo::DeviceGuard guard(ctx->device);
+    if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
+    DevicePlan d;
+    st = upload_plan(ctx, plan, stream, &d);
+    if (st != EVO_OK) return st;
+    const uint32_t n_ctas = static_cast<uint32_t>(plan.ranges.size());
+    if (n_ctas > 0) {
+        generated_pass1<<<n_ctas, kThreads, 0, stream>>>(round_keys(seed), d.sets, d.members, d.ranges, d.parts);
+        ctx->launches += 1;
+        EVO_CUDA_TRY(ctx, cudaGetLastError());
+    }
+    return finish_exact(ctx, d, n_desc, results, group_pass, n_group, stream);
 }
