@@ -384,6 +384,47 @@ def measure_config(evo, ctx, name, device, peak, reps):
     return out
 
 
+def measure_generated(evo, ctx, device, peak, log2_n=28, reps=10):
+    """evo_validate_generated (reference regenerated in the kernel) against the two-step route evo_gen_inputs(raw words)
+    + evo_validate_exact, for one candidate and for sixteen candidates of 2^log2_n words each."""
+    n = 1 << log2_n
+    ref = torch.empty(n, dtype=torch.int32, device=device)
+    out = {"elements_per_tensor": n, "dtype": "u32 words compared as int32", "reps": reps}
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    evo.evo_gen_inputs(7, 0, evo.EVO_U32, n, ref, ctx=ctx)
+    for k in (1, 16):
+        cands = [ref.clone() for _ in range(k)]
+        cands[-1][n // 3] += 1                                  # one wrong element in the last candidate
+        fused_ms = timed(lambda: evo.evo_validate_generated(7, cands, offsets=0, dtype=evo.EVO_I32, ctx=ctx))
+
+        def two_step():
+            evo.evo_gen_inputs(7, 0, evo.EVO_U32, n, ref, ctx=ctx)
+            evo.evo_validate_exact(cands, [ref] * k, ctx=ctx)
+        two_ms = timed(two_step)
+        got = evo.exact_to_numpy(evo.evo_validate_generated(7, cands, offsets=0, dtype=evo.EVO_I32, ctx=ctx)[0])
+        assert got["n_mismatch"].sum() == 1 and got["n_mismatch"][-1] == 1, "fused check is wrong"
+        cand_bytes = 4 * n * k
+        out["k%d" % k] = {"fused_ms": fused_ms, "generate_then_check_ms": two_ms, "speedup": two_ms / fused_ms,
+                          "fused_candidate_gbs": cand_bytes / (fused_ms * 1e-3) / 1e9,
+                          "fused_frac_of_peak": cand_bytes / (fused_ms * 1e-3) / 1e9 / peak}
+        del cands
+    del ref
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import paper_2510_03760_b200 as evo
 
@@ -418,11 +459,21 @@ def run_ours(args):
     # the pointer and descriptor arrays of the population are marshalled once: the tensors do not move between steps
     prepared = evo.Prepared(cands, refs, groups, n_group)
 
+    # The test inputs of the next case do not depend on this case's check: they are generated on a second stream
+    # (a context of its own), launched after the check so that the check's persistent CTAs are resident first and the
+    # generator fills the room they leave.  The timed region ends only when both streams have drained.
+    main_stream = torch.cuda.current_stream(device)
+    side_stream = torch.cuda.Stream(device) if args.overlap_gen else main_stream
+    gen_ctx = evo.Context(local_rank) if args.overlap_gen else ctx
+
     def step(i, ev=None):
-        evo.evo_gen_inputs(1000 + i, 0, evo.EVO_F32, n_gen, gen_buf, ctx=ctx)
+        if not args.overlap_gen:
+            evo.evo_gen_inputs(1000 + i, 0, evo.EVO_F32, n_gen, gen_buf, ctx=ctx)
         if ev is not None:
             ctx.set_timing_events(ev[0], ev[1])
         evo.evo_validate(prepared, None, pop.atol, pop.rtol, results=results, group_pass=gpass, ctx=ctx)
+        if args.overlap_gen:
+            evo.evo_gen_inputs(1000 + i, 0, evo.EVO_F32, n_gen, gen_buf, stream=side_stream, ctx=gen_ctx)
         evo.evo_fitness(pop.times, pop.base_times, gpass, out=fits, ctx=ctx)
 
     for i in range(max(args.warmup, 3)):
@@ -438,15 +489,16 @@ def run_ours(args):
 
     sampler = ClockSampler(torch.cuda._get_nvml_device_index(local_rank) if hasattr(torch.cuda, "_get_nvml_device_index") else local_rank)
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches_before = ctx.launches
+    launches_before, gen_launches_before = ctx.launches, gen_ctx.launches
     with sampler:
         barrier()
         start.record()
         for i in range(args.steps):
             step(i, kern_events[i])
+        main_stream.wait_stream(side_stream)
         stop.record()
         barrier()
-    launches = ctx.launches - launches_before
+    launches = ctx.launches - launches_before + (gen_ctx.launches - gen_launches_before if gen_ctx is not ctx else 0)
     total_ms = start.elapsed_time(stop)
     kern_ms = [a.elapsed_time(b) for a, b in kern_events]
     if distributed:
@@ -533,6 +585,7 @@ def run_ours(args):
 
     # the other synthetic populations, with the main one out of the way
     config = config_keys(args.workload, n_gen, len(cands), n_group, int(pop.times.shape[1]), alg_bytes, world)
+    streams = "evo_gen_inputs on a second stream, concurrent with evo_validate" if args.overlap_gen else "one stream"
     candidate_bytes = pop.candidate_bytes()
     per_config = None
     if args.per_config:
@@ -542,6 +595,7 @@ def run_ours(args):
         for name, reps in (("config1", 200), ("config2", 200), ("config3", 100), ("config5", 20)):
             if name != args.workload:
                 per_config[name] = measure_config(evo, ctx, name, device, peak, reps)
+        per_config["fused_generate_compare"] = measure_generated(evo, ctx, device, peak)
 
     cpu = cpu_many = None
     if not args.no_cpu_baseline:
@@ -566,7 +620,7 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "n_gpus_requested": args.gpus, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config, "streams": streams,
         "candidates_per_s": cand_per_s, "frac_of_hbm_peak": value / world / peak,
         "frac_of_datasheet_hbm": value / world / DATASHEET_HBM_GBS,
         "candidate_bytes_gbs": world * candidate_bytes / (ms_per_step * 1e-3) / 1e9, "plan": plan_info,
@@ -598,6 +652,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap-gen", dest="overlap_gen", action="store_false",
+                    help="generate the test inputs on the main stream, before the check, instead of on a second stream")
     ap.add_argument("--no-per-config", dest="per_config", action="store_false",
                     help="skip the figures of the other synthetic populations (configs 1, 2, 3, 5)")
     ap.add_argument("--log2-elems", type=int, default=None,
