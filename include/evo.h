@@ -154,6 +154,12 @@ typedef struct {
  *             descriptors with .group == g (1 for a group without descriptors).
  * Tensors need only element alignment; 16-byte aligned tensors take the fast path.
  * The host arrays are consumed before the call returns.  n_desc == 0 is legal.
+ * A call whose pointer and descriptor arrays, reference, dtype, groups and stream equal those of
+ * the call before it on the same context (an evaluation loop that reuses its buffers for every
+ * test case) reuses that call's schedule, which is still in device memory, and only launches the
+ * kernels; the tensors are read again, the tolerances may differ.  Schedules of up to 32 KiB
+ * (a few hundred tensors) reach the device as kernel arguments, larger ones by a copy from a
+ * pinned block of the context.
  * Errors: EVO_ERR_ARG, EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_WORKSPACE, EVO_ERR_CUDA.
  */
 EVO_API int evo_validate(evo_ctx* ctx, const void* const* cand_ptrs /* host array of device ptrs */,

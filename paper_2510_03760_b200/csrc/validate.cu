@@ -49,6 +49,7 @@ namespace {
 using namespace evo;
 
 constexpr int kCtasPerSm = 2;
+constexpr int kCtasPerSm16 = 3;                     // for populations of 16-bit tensors only
 constexpr int kStages = 6;                          // ring depth per CTA
 constexpr int kStageBytes = kTileElems * 4;         // 16 KiB: one fp32 tile (a 16-bit tile uses half)
 constexpr size_t kRingBytes = static_cast<size_t>(kStages) * kStageBytes;
@@ -141,12 +142,13 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 struct Ring {
     uint32_t full0, empty0;     // shared-memory addresses of full[0], empty[0]
     uint32_t data0;             // ... and of stage 0
+    uint32_t stage_bytes;       // 16 KiB, or 8 KiB in the kernel for populations of 16-bit tensors only
     uint32_t stage = 0, phase = 0;
     bool dead = false;          // this warp has given up (warp-uniform)
     volatile int* abort_flag;
     __device__ __forceinline__ uint32_t full() const { return full0 + 8u * stage; }
     __device__ __forceinline__ uint32_t empty() const { return empty0 + 8u * stage; }
-    __device__ __forceinline__ uint32_t data() const { return data0 + static_cast<uint32_t>(kStageBytes) * stage; }
+    __device__ __forceinline__ uint32_t data() const { return data0 + stage_bytes * stage; }
     __device__ __forceinline__ void advance() { if (++stage == kStages) { stage = 0; phase ^= 1u; } }
 };
 
@@ -618,8 +620,10 @@ __device__ __forceinline__ uint32_t producer_loop(const SetRec* __restrict__ set
     return issued;
 }
 
-__global__ void __launch_bounds__(kBlock, kCtasPerSm)
-validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
+// The body of the first pass.  kOnly16: the population holds fp16/bf16 tensors only; the fp32 path (more
+// registers, 16 KiB stages) is then left out, which lets a third CTA share the SM (see validate_pass1_16bit).
+template <bool kOnly16>
+__device__ __forceinline__ void pass1_body(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
                const CtaRange* __restrict__ ranges, Acc* __restrict__ partials, float atol, float rtol,
                uint32_t* __restrict__ status, const uint32_t* __restrict__ seeds /* optional: see seed_kernel */,
                unsigned long long* __restrict__ cta_times /* optional: %globaltimer at start and end of every CTA */) {
@@ -640,7 +644,7 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
     }
     __syncthreads();
     // Up to here nothing depended on earlier work in the stream; the plan, the seeds and the tensors do.
-    grid_dependents_may_launch();
+    if (!kOnly16) grid_dependents_may_launch();
     grid_dependency_wait();
     if (cta_times && threadIdx.x == 0) cta_times[2 * blockIdx.x] = global_ns();
     const CtaRange rg = ranges[blockIdx.x];
@@ -648,6 +652,7 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
     g.full0 = smem_u32(&s_full[0]);
     g.empty0 = smem_u32(&s_empty[0]);
     g.data0 = smem_u32(s_ring);
+    g.stage_bytes = kOnly16 ? kStageBytes / 2 : kStageBytes;
     g.abort_flag = &s_abort;
     uint32_t issued = 0;
 
@@ -668,7 +673,7 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
                 s_mr[threadIdx.x] = seeds ? seeds[S.member_off + threadIdx.x] : 0u;
             }
             consumer_bar();
-            if (S.dtype == EVO_F32) run_set<EVO_F32>(S, sp, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
+            if (!kOnly16 && S.dtype == EVO_F32) run_set<EVO_F32>(S, sp, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
             else if (S.dtype == EVO_F16) run_set<EVO_F16>(S, sp, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
             else run_set<EVO_BF16>(S, sp, atol, rtol, s_acc, s_mr, s_cand, g, warp, lane);
             consumer_bar();
@@ -686,6 +691,10 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
             consumer_bar();
         }
     }
+    // With three CTAs per SM the register file is full: kernels that start early would only take the places of
+    // this kernel's own CTAs and wait there (measured: 20 us lost per call on 128 x 2 MiB); they may start once
+    // this CTA's work is done.
+    if (kOnly16) grid_dependents_may_launch();
     __syncthreads();
     if (s_abort) {
         // A wait ran out.  Before the CTA gives its shared memory back, let the copies that
@@ -703,6 +712,23 @@ validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ me
         if (threadIdx.x == 0) atomicOr(status, 1u);
     }
     if (cta_times && threadIdx.x == 0) cta_times[2 * blockIdx.x + 1] = global_ns();
+}
+
+__global__ void __launch_bounds__(kBlock, kCtasPerSm)
+validate_pass1(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
+               const CtaRange* __restrict__ ranges, Acc* __restrict__ partials, float atol, float rtol,
+               uint32_t* __restrict__ status, const uint32_t* __restrict__ seeds, unsigned long long* __restrict__ cta_times) {
+    pass1_body<false>(sets, members, ranges, partials, atol, rtol, status, seeds, cta_times);
+}
+
+// The same pass for populations without fp32 tensors.  16-bit tiles are 8 KiB, so the ring is half as large, and
+// the 16-bit path needs fewer registers: three CTAs (27 warps) share an SM instead of two, which is what a pass
+// bound by instruction issue rather than by memory (two bytes per element for the same arithmetic) can use.
+__global__ void __launch_bounds__(kBlock, kCtasPerSm16)
+validate_pass1_16bit(const SetRec* __restrict__ sets, const MemberRec* __restrict__ members,
+                     const CtaRange* __restrict__ ranges, Acc* __restrict__ partials, float atol, float rtol,
+                     uint32_t* __restrict__ status, const uint32_t* __restrict__ seeds, unsigned long long* __restrict__ cta_times) {
+    pass1_body<true>(sets, members, ranges, partials, atol, rtol, status, seeds, cta_times);
 }
 
 // Warm start for the filter of max d/|r|.  A CTA that begins a run knows no maximum for its
@@ -929,6 +955,7 @@ struct ChainArgs {
     uint32_t* group_pass;
     uint64_t n_group;
     bool pdl;
+    bool only16;                      // no fp32 tensor in the population: the three-CTAs-per-SM kernel
     cudaEvent_t ev_start, ev_stop;    // optional: around the first pass
 };
 
@@ -947,7 +974,8 @@ cudaError_t launch_chain(uint32_t n_members, uint32_t n_ctas, const ChainArgs& a
     }
     if (a.ev_start && (e = cudaEventRecord(a.ev_start, stream)) != cudaSuccess) return e;
     if (n_ctas > 0) {
-        e = evo::launch(validate_pass1, dim3(n_ctas), dim3(kBlock), kRingBytes, stream, a.pdl, d_sets, d_members, d_ranges,
+        e = evo::launch(a.only16 ? validate_pass1_16bit : validate_pass1, dim3(n_ctas), dim3(kBlock),
+                        a.only16 ? kRingBytes / 2 : kRingBytes, stream, a.pdl, d_sets, d_members, d_ranges,
                         a.d_parts, a.atol, a.rtol, a.d_status, static_cast<const uint32_t*>(a.d_seeds && n_members ? a.d_seeds : nullptr),
                         a.d_cta_times);
         if (e != cudaSuccess) return e;
@@ -1003,7 +1031,12 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     if (!(atol >= 0.f) || !(rtol >= 0.f) || std::isinf(atol) || std::isinf(rtol))
         return evo::fail(ctx, EVO_ERR_ARG, "%s: atol and rtol must be finite and >= 0", who);
     if (n_desc > 0 && (!cand_ptrs || !descs)) return evo::fail(ctx, EVO_ERR_ARG, "%s: cand_ptrs and descs must not be NULL", who);
-    const uint32_t max_ctas = static_cast<uint32_t>(ctx->sm_count) * kCtasPerSm;
+    bool only16 = n_desc > 0;
+    for (uint64_t i = 0; i < n_desc && only16; ++i) {
+        const int dt = descs[i].dtype == -1 ? dtype : descs[i].dtype;
+        only16 = dt == EVO_F16 || dt == EVO_BF16;
+    }
+    const uint32_t max_ctas = static_cast<uint32_t>(ctx->sm_count) * (only16 ? kCtasPerSm16 : kCtasPerSm);
 
     evo::DeviceGuard guard(ctx->device);
     if (guard.err != cudaSuccess) return evo::fail_cuda(ctx, guard.err, "cudaSetDevice");
@@ -1077,6 +1110,8 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     if (n_ctas > 0 && !ctx->pass1_ready) {
         EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(validate_pass1, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                static_cast<int>(kRingBytes)));
+        EVO_CUDA_TRY(ctx, cudaFuncSetAttribute(validate_pass1_16bit, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               static_cast<int>(kRingBytes / 2)));
         ctx->pass1_ready = true;
     }
     ChainArgs a{};
@@ -1089,6 +1124,7 @@ int validate_device(evo_ctx* ctx, const void* const* cand_ptrs, const void* ref_
     a.atol = atol; a.rtol = rtol;
     a.results = results; a.group_pass = group_pass; a.n_group = n_group;
     a.pdl = ctx->pdl;
+    a.only16 = only16;
     a.ev_start = ev_start; a.ev_stop = ev_stop;
     const cudaError_t e = launch_chain(n_members, n_ctas, a, stream, &ctx->launches);
     if (e != cudaSuccess) return evo::fail_cuda(ctx, e, "kernel launch");

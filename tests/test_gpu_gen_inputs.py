@@ -70,6 +70,20 @@ def test_large_fill_statistics_and_sampled_parity(evo):
         assert np.abs(ordered(got) - ordered(want)).max() <= 4
 
 
+def test_fill_of_the_largest_configuration_in_full(evo):
+    """2^28 fp32 normals, the test-input tensor of the largest synthetic configuration, in the launch shape the
+    benchmark uses: every element against the oracle, in pieces of 2^24 (about 20 s of oracle time)."""
+    n, piece = 1 << 28, 1 << 24
+    out = torch.empty(n, dtype=torch.float32, device="cuda")
+    evo.evo_gen_inputs(1000, 0, evo.EVO_F32, n, out)
+    worst = 0
+    for start in range(0, n, piece):
+        got = out[start:start + piece].cpu().numpy()
+        want = oracle.gen_inputs(1000, start, oracle.F32, piece)
+        worst = max(worst, int(np.abs(ordered(got) - ordered(want)).max()))
+    assert worst <= 4, worst
+
+
 def test_argument_errors(evo):
     out = torch.zeros(16, dtype=torch.float32, device="cuda")
     L, ctx = evo.load_library(), evo.default_context(0)
