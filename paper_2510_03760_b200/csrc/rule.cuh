@@ -27,7 +27,6 @@ template <int DT> struct Elem;
 template <> struct Elem<EVO_F32> {
     static constexpr int kPerVec = 4;
     static constexpr int kVecs = kEpt / 4;          // 16-byte vectors per thread per tile
-    static constexpr int kTolGroups = 1;            // groups of a thread's elements with a smallest tolerance of their own
     using T = float;
     static __device__ __forceinline__ float at(const uint4& v, int i) {
         return __uint_as_float(i == 0 ? v.x : i == 1 ? v.y : i == 2 ? v.z : v.w);
@@ -37,7 +36,6 @@ template <> struct Elem<EVO_F32> {
 template <> struct Elem<EVO_F16> {
     static constexpr int kPerVec = 8;
     static constexpr int kVecs = kEpt / 8;
-    static constexpr int kTolGroups = 1;
     using T = __half;
     static __device__ __forceinline__ float at(const uint4& v, int i) {
         const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;
@@ -49,7 +47,6 @@ template <> struct Elem<EVO_F16> {
 template <> struct Elem<EVO_BF16> {
     static constexpr int kPerVec = 8;
     static constexpr int kVecs = kEpt / 8;
-    static constexpr int kTolGroups = 1;
     using T = __nv_bfloat16;
     static __device__ __forceinline__ float at(const uint4& v, int i) {
         const uint32_t w = (i >> 1) == 0 ? v.x : (i >> 1) == 1 ? v.y : (i >> 1) == 2 ? v.z : v.w;

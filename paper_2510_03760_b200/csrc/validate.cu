@@ -266,10 +266,9 @@ constexpr float kInf = __builtin_huge_valf();
 // One full, 16-byte aligned tile: reference into registers once, then every member.
 //
 // Fast path per element, valid when c and r are finite and d does not overflow: d = |c - r|,
-// its maximum and its square; mismatches are counted only in a group of elements (Elem::kTolGroups per
-// thread: one group of 16 measured fastest for every type) whose largest d exceeds the smallest
-// tolerance of the group.  With atol, rtol >= 0 and finite data c == r implies d = 0 <= tol, so the
-// equality clause needs no test here.
+// its maximum and its square; mismatches are counted only for a thread whose largest d exceeds the
+// smallest tolerance of its 16 elements.  With atol, rtol >= 0 and finite data c == r implies
+// d = 0 <= tol, so the equality clause needs no test here.
 // The quotient d/|r| is not formed.  With m the running maximum of the quotient (a binary32 value),
 // fl(d/|r|) > m implies d/|r| > m (rounding is monotone and m is representable), hence
 // d > m*|r| >= RZ(m*|r|): the test d > RZ(m*|r|) never misses a new maximum, and an element that only
@@ -279,8 +278,6 @@ template <int DT>
 __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, float atol, float rtol, Acc (*s_acc)[kWarps],
                                           uint32_t* s_mr, const void* const* s_cand, Ring& g, int warp, int lane) {
     using E = Elem<DT>;
-    constexpr int kGroups = E::kTolGroups;          // groups of elements with a smallest tolerance of their own
-    constexpr int kPerGroup = kEpt / kGroups;
     if (g.dead) return;
     float r[kEpt];
     {
@@ -291,17 +288,15 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
 #pragma unroll
             for (int e = 0; e < E::kPerVec; ++e) r[v * E::kPerVec + e] = E::at(rv[v], e);
     }
-    // The smallest tolerance among a group's reference elements: tol = atol + rtol*|r| does not decrease with |r|
-    // (each rounding is monotone), so it is the tolerance of the smallest |r|.  A member whose largest difference
-    // over the group stays within it has no mismatch there, and none is counted element by element.
-    float tolmin[kGroups];
+    // The smallest tolerance among this thread's 16 reference elements: tol = atol + rtol*|r| does not decrease
+    // with |r| (each rounding is monotone), so it is the tolerance of the smallest |r|.  A member whose largest
+    // difference over these elements stays within it has no mismatch here, and none is counted element by element.
+    // (Finer groups - a tolerance per 16-byte vector - and a walk shared out over the warp were measured: no gain on
+    // data with values on the boundary, a loss on candidates that are wrong everywhere.)
+    float armin = kInf;
 #pragma unroll
-    for (int q = 0; q < kGroups; ++q) {
-        float armin = kInf;
-#pragma unroll
-        for (int e = 0; e < kPerGroup; ++e) armin = fminf(armin, fabsf(r[q * kPerGroup + e]));
-        tolmin[q] = __fadd_rn(atol, __fmul_rn(rtol, armin));
-    }
+    for (int e = 0; e < kEpt; ++e) armin = fminf(armin, fabsf(r[e]));
+    const float tolmin = __fadd_rn(atol, __fmul_rn(rtol, armin));
     const uint64_t vec0 = t * (kTileElems / E::kPerVec) + threadIdx.x;   // this thread's first vector of the tile
 #pragma unroll 1
     for (int k = 0; k < K; ++k) {
@@ -312,44 +307,35 @@ __device__ __forceinline__ void fast_tile(const void* ref, int K, uint64_t t, fl
         // value only makes the filter fire more often.
         const float m = __uint_as_float(*reinterpret_cast<volatile uint32_t*>(&s_mr[k]));
         uint32_t cnt = 0;
-        float sse = 0.f;
-        float mag[kGroups];
+        float ma = 0.f, sse = 0.f;
         bool trig = false;
 #pragma unroll
-        for (int q = 0; q < kGroups; ++q) {
-            mag[q] = 0.f;
+        for (int v = 0; v < E::kVecs; ++v)
 #pragma unroll
-            for (int e = 0; e < kPerGroup; e += 2) {
-                const int i = q * kPerGroup + e;
-                const float d0 = fabsf(__fsub_rn(E::at(cv[i / E::kPerVec], i % E::kPerVec), r[i]));
-                const float d1 = fabsf(__fsub_rn(E::at(cv[(i + 1) / E::kPerVec], (i + 1) % E::kPerVec), r[i + 1]));
-                mag[q] = max3(mag[q], d0, d1);
+            for (int e = 0; e < E::kPerVec; e += 2) {
+                const int i = v * E::kPerVec + e;
+                const float d0 = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
+                const float d1 = fabsf(__fsub_rn(E::at(cv[v], e + 1), r[i + 1]));
+                ma = max3(ma, d0, d1);
                 sse = fmaf(d0, d0, sse);
                 sse = fmaf(d1, d1, sse);
                 trig |= d0 > __fmul_rz(m, fabsf(r[i]));
                 trig |= d1 > __fmul_rz(m, fabsf(r[i + 1]));
             }
-        }
-        float ma = mag[0];
-#pragma unroll
-        for (int q = 1; q < kGroups; ++q) ma = fmaxf(ma, mag[q]);
         // The fast numbers do not stand if something was NaN/Inf or overflowed (the sum of
         // squares is then NaN/Inf) or if every d is so small that d^2 underflows in binary32.
         const bool redo = !(sse < kInf) || (ma < 9.094947017729282e-13f /* 2^-40 */ && ma > 0.f);
-        if (!redo) {
+        if (ma > tolmin && !redo) {
+            // some difference may exceed its tolerance: count, element by element
 #pragma unroll
-            for (int q = 0; q < kGroups; ++q) {
-                if (mag[q] > tolmin[q]) {
-                    // some difference of this group may exceed its tolerance: count, element by element
+            for (int v = 0; v < E::kVecs; ++v)
 #pragma unroll
-                    for (int e = 0; e < kPerGroup; ++e) {
-                        const int i = q * kPerGroup + e;
-                        const float d = fabsf(__fsub_rn(E::at(cv[i / E::kPerVec], i % E::kPerVec), r[i]));
-                        const float tol = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r[i])));
-                        cnt += (d > tol) ? 1u : 0u;
-                    }
+                for (int e = 0; e < E::kPerVec; ++e) {
+                    const int i = v * E::kPerVec + e;
+                    const float d = fabsf(__fsub_rn(E::at(cv[v], e), r[i]));
+                    const float tol = __fadd_rn(atol, __fmul_rn(rtol, fabsf(r[i])));
+                    cnt += (d > tol) ? 1u : 0u;
                 }
-            }
         }
         float mt = m;
         float lo = m;
