@@ -69,7 +69,7 @@ def measured_peak():
 # DRAM traffic of validate_pass1 as counted by ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a reduced
 # config 4 (2^24 elements per tensor), per algorithmic byte (the capture is summarised under profiles/).
 # It stands only for the kernel sources it was captured on: their hash is checked, and a mismatch reports null.
-NCU_TRAFFIC = {"dram_bytes_per_algorithmic_byte": 1.006, "sources_sha1": "bb401ccbd21d8636dbe08b0724bdf0740fec5a78"}
+NCU_TRAFFIC = {"dram_bytes_per_algorithmic_byte": 1.0054, "sources_sha1": "f2bc9e94633325e6f6401f899b16075f308976c0"}
 
 
 def kernel_sources_sha1():
@@ -501,6 +501,18 @@ def run_ours(args):
     launches = ctx.launches - launches_before + (gen_ctx.launches - gen_launches_before if gen_ctx is not ctx else 0)
     total_ms = start.elapsed_time(stop)
     kern_ms = [a.elapsed_time(b) for a, b in kern_events]
+
+    # The main kernel by itself: a few more steps, outside the timed region, with nothing beside it on the device
+    # (in the timed region the generator runs concurrently and takes its share of issue slots and of HBM writes).
+    kern_alone_ms = None
+    if args.overlap_gen:
+        alone = kern_events[: min(20, len(kern_events))]
+        torch.cuda.synchronize()
+        for a, b in alone:
+            ctx.set_timing_events(a, b)
+            evo.evo_validate(prepared, None, pop.atol, pop.rtol, results=results, group_pass=gpass, ctx=ctx)
+        torch.cuda.synchronize()
+        kern_alone_ms = [a.elapsed_time(b) for a, b in alone]
     if distributed:
         t = torch.tensor([total_ms], device=device, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -578,6 +590,14 @@ def run_ours(args):
                 "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms_avg": kern_avg_ms,
                 "kernel_ms_min": min(kern_ms), "kernel_ms_max": max(kern_ms)}
 
+    if kern_alone_ms:
+        alone_avg = sum(kern_alone_ms) / len(kern_alone_ms)
+        roofline["kernel_ms_alone"] = alone_avg
+        roofline["achieved_alone"] = alg_bytes / (alone_avg * 1e-3) / 1e9
+        roofline["frac_alone"] = roofline["achieved_alone"] / peak
+        roofline["concurrency"] = ("achieved/frac: the kernel as it runs in the timed region, with evo_gen_inputs concurrent on a "
+                                   "second stream (1 GiB of HBM writes and its arithmetic beside it); *_alone: %d more launches after "
+                                   "the timed region with nothing else on the device" % len(kern_alone_ms))
     roofline["datasheet_peak"] = DATASHEET_HBM_GBS
     roofline["frac_of_datasheet"] = achieved / DATASHEET_HBM_GBS
     roofline["note"] = ("frac is against the measured copy bandwidth of this pool's B200s (a read+write copy; a read-only stream "
