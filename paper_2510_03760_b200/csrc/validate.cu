@@ -12,7 +12,9 @@
 //   plan (host)   tensors with the same (reference, n, dtype) form a set of up to kMaxK
 //                 members; the flat list of (set, tile) items, weighted by the tiles they
 //                 move, is cut into one contiguous range per CTA (a fixed cut: no work
-//                 queue, no atomics, results reproducible run to run).
+//                 queue, no atomics, results reproducible run to run).  A small plan reaches
+//                 the device as kernel arguments (plan_store), a large one by one copy; a call
+//                 with the arguments of the call before reuses the plan that is already there.
 //   pass 1        persistent CTAs walk their range.  A producer warp streams the tiles
 //                 (reference, then each member) into a ring of shared-memory stages with
 //                 bulk asynchronous copies that complete on mbarriers; eight consumer warps
@@ -22,7 +24,11 @@
 //                 memory.  When a CTA leaves a set it writes one partial record per member.
 //   pass 2        one warp per tensor folds the partial records of the CTAs that touched
 //                 it, in a fixed order, and writes the evo_result.
-//   verdict       one thread per candidate id ANDs the verdicts of its tensors.
+//   verdict       one thread per candidate id ANDs the verdicts of its tensors (inside
+//                 pass 2 when one CTA holds every tensor).
+//
+// Every kernel is launched so that it may begin under the tail of its predecessor
+// (programmatic dependent launch) and waits for it before touching global memory.
 //
 // Every wait on an mbarrier is bounded: after kWaitLimitNs the CTA stops working, lets its
 // outstanding copies land, raises the status word and returns; pass 2 then marks every

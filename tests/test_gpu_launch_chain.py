@@ -127,3 +127,22 @@ def test_whole_step_back_to_back_matches_the_oracle(evo):
     wz = oracle.gen_inputs(29, 0, oracle.F32, 20000)
     from parity import ordered
     assert np.abs(ordered(z) - ordered(wz)).max() <= 4
+
+
+def test_per_cta_clocks_cover_every_cta_and_lie_inside_the_call(evo):
+    """evo_debug_cta_timing: one (begin, end) pair of the GPU's nanosecond clock per persistent CTA of the main kernel;
+    begin <= end, all within a few milliseconds of each other, as many pairs as the plan has CTAs; off again afterwards."""
+    ctx = evo.Context(0)
+    pop = workloads.config5("cpu", n_cand=200, log2_min=8.0, log2_max=17.0, trials=4)
+    cands, refs, groups = _dev(pop)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    ctx.cta_timing(True)
+    res, gp = evo.evo_validate(cands, refs, pop.atol, pop.rtol, groups=groups, n_group=pop.n_group, ctx=ctx)
+    t = ctx.read_cta_times()
+    info = evo.plan_inspect(cands, refs, 2 * sms)
+    assert len(t) == info["n_ctas"] and len(t) > 0
+    assert (t[:, 1] >= t[:, 0]).all() and int(t[:, 1].max() - t[:, 0].min()) < 50_000_000
+    assert_results_equal(evo.results_to_numpy(res), oracle_population(pop)[0], "with per-CTA clocks")
+    ctx.cta_timing(False)
+    evo.evo_validate(cands, refs, pop.atol, pop.rtol, groups=groups, n_group=pop.n_group, ctx=ctx)
+    assert len(ctx.read_cta_times()) == 0
