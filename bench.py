@@ -603,12 +603,30 @@ def run_ours(args):
     roofline["note"] = ("frac is against the measured copy bandwidth of this pool's B200s (a read+write copy; a read-only stream "
                         "can exceed it a little); frac_of_datasheet is against the nominal %d GB/s" % DATASHEET_HBM_GBS)
 
+    # The generator is bound by plain arithmetic: 56 lane-slots per normal (ncu, smsp__inst_executed x 32 / normals)
+    # against the issue peak of the part, SMs x 4 schedulers x 32 lanes x the SM clock.
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    g0.record()
+    for i in range(5):
+        evo.evo_gen_inputs(4000 + i, 0, evo.EVO_F32, n_gen, gen_buf, ctx=ctx)
+    g1.record()
+    torch.cuda.synchronize()
+    gen_ms = g0.elapsed_time(g1) / 5
+    props = torch.cuda.get_device_properties(device)
+    sm_mhz_max = sampler.max_mhz or 1965
+    issue_peak = props.multi_processor_count * 4 * 32 * sm_mhz_max * 1e6 / 1e12
+    gen_info = {"kernel": "gen_kernel<f32>", "bound": "alu", "normals": n_gen, "kernel_ms": gen_ms,
+                "lane_slots_per_normal": 56, "achieved": 56 * n_gen / (gen_ms * 1e-3) / 1e12, "peak": issue_peak,
+                "unit": "T lane-slots/s", "frac": 56 * n_gen / (gen_ms * 1e-3) / 1e12 / issue_peak,
+                "peak_kind": "SMs x 4 schedulers x 32 lanes x max SM clock"}
+
     # the other synthetic populations, with the main one out of the way
     config = config_keys(args.workload, n_gen, len(cands), n_group, int(pop.times.shape[1]), alg_bytes, world)
     streams = "evo_gen_inputs on a second stream, concurrent with evo_validate" if args.overlap_gen else "one stream"
     candidate_bytes = pop.candidate_bytes()
     per_config = None
-    if args.per_config:
+    if args.per_config and world == 1:
         del prepared, cands, refs, pop, gen_buf
         torch.cuda.empty_cache()
         per_config = {}
@@ -618,7 +636,7 @@ def run_ours(args):
         per_config["fused_generate_compare"] = measure_generated(evo, ctx, device, peak)
 
     cpu = cpu_many = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and world == 1:           # the baseline legs belong to the one-GPU run
         # about 10 s of single-thread work: the sample of the reference arm, several passes
         sample = OracleSample(args.workload, ORACLE_SAMPLE_LOG2[0], ORACLE_SAMPLE_LOG2[1])
         sample.run()
@@ -645,7 +663,7 @@ def run_ours(args):
         "frac_of_datasheet_hbm": value / world / DATASHEET_HBM_GBS,
         "candidate_bytes_gbs": world * candidate_bytes / (ms_per_step * 1e-3) / 1e9, "plan": plan_info,
         "clocks": sampler.summary(), "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": roofline, "cpu_baseline": cpu, "cpu_baseline_all_cores": cpu_many, "per_config": per_config,
+        "roofline": roofline, "roofline_generator": gen_info, "cpu_baseline": cpu, "cpu_baseline_all_cores": cpu_many, "per_config": per_config,
     }
     print(json.dumps(line))
     if distributed:

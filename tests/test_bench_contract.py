@@ -76,6 +76,10 @@ def test_gpu_arm_prints_one_json_line_with_roofline_e2e_and_cpu_baseline():
     r = j["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 0 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert r["frac_of_datasheet"] < r["frac"] and r["datasheet_peak"] == 7700.0
+    assert r["frac_alone"] > 0 and r["kernel_ms_alone"] > 0              # the kernel with nothing beside it, after the timed region
+    gen = j["roofline_generator"]
+    assert gen["bound"] == "alu" and 0 < gen["frac"] < 1.2 and abs(gen["frac"] - gen["achieved"] / gen["peak"]) < 1e-9
+    assert j["streams"].startswith("evo_gen_inputs on a second stream")
     e = j["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] >= j["config"]["algorithmic_bytes_per_step"] and e["d2h_bytes_per_step"] > 0
     c = j["cpu_baseline"]
