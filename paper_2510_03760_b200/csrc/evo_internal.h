@@ -22,7 +22,7 @@ struct evo_ctx {
     void* d_stage = nullptr;     size_t d_stage_bytes = 0;      // tensors of the *_host calls
     void* d_seeds = nullptr;     size_t d_seeds_bytes = 0;      // per tensor: warm start of the max d/|r| filter
     void* d_feedback = nullptr;  size_t d_feedback_bytes = 0;   // per-chunk counts of evo_mismatch_sample
-    void* d_small = nullptr;                                   // 256 bytes: baseline median (0..127), status word (128)
+    void* d_small = nullptr;                                   // 256 bytes: summary scratch (64..), status word (128)
     bool pass1_ready = false;                                  // the first pass's shared-memory size has been set
     cudaEvent_t plan_consumed = nullptr;                       // the last plan upload has been read
     bool plan_in_flight = false;
