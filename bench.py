@@ -43,6 +43,7 @@ WORKLOAD_NOTES = {
     "config3": "64 fp16 + 64 bf16 candidates x 2^20 elements, one reference per dtype",
     "config5": "1024 candidates, 1-3 tensors each, 2^10..2^24 elements, fp32/fp16/bf16, own references",
     "config2": "8 fp32 candidates x 262144 elements sharing one reference (fits in L2)",
+    "clean16": "8 bf16 candidates x 2^26 elements sharing one reference, noise far below the tolerance",
 }
 
 
@@ -148,7 +149,7 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- oracle arm
 FULL_SHAPE = {"config4": dict(n=1 << 28, k=16), "config3": dict(n=1 << 20, k=128), "config2": dict(n=1 << 18, k=8),
-              "config1": dict(n=1 << 12, k=1)}
+              "config1": dict(n=1 << 12, k=1), "clean16": dict(n=1 << 26, k=8)}
 FULL_TRIALS = {"config1": 5}
 
 
@@ -166,6 +167,8 @@ class OracleSample:
                 pop = workloads.config3("cpu", n=n_s, k_per_dtype=2)
             elif workload == "config1":
                 pop = workloads.config1("cpu")
+            elif workload == "clean16":
+                pop = workloads.clean16("cpu", n=n_s, k=4)
             else:
                 pop = workloads.config2("cpu", n=n_s, k=4)
             self.scale_val = (n_full * k_full) / float(n_s * len(pop.tensors))
@@ -207,7 +210,8 @@ ORACLE_SAMPLE_LOG2 = (24, 22)
 
 
 def full_algorithmic_bytes(workload):
-    known = {"config4": 17 * (1 << 30), "config3": 130 * (1 << 21), "config2": 9 * (1 << 20), "config1": 2 * (1 << 14)}
+    known = {"config4": 17 * (1 << 30), "config3": 130 * (1 << 21), "config2": 9 * (1 << 20), "config1": 2 * (1 << 14),
+             "clean16": 9 * (1 << 27)}
     return known.get(workload, int(2048 * 1.73e6 * 3 * 2))
 
 
@@ -630,7 +634,7 @@ def run_ours(args):
         del prepared, cands, refs, pop, gen_buf
         torch.cuda.empty_cache()
         per_config = {}
-        for name, reps in (("config1", 200), ("config2", 200), ("config3", 100), ("config5", 20)):
+        for name, reps in (("config1", 200), ("config2", 200), ("config3", 100), ("config5", 20), ("clean16", 20)):
             if name != args.workload:
                 per_config[name] = measure_config(evo, ctx, name, device, peak, reps)
         per_config["fused_generate_compare"] = measure_generated(evo, ctx, device, peak)

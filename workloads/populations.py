@@ -190,6 +190,22 @@ def config5(device="cpu", n_cand=1024, log2_min=10.0, log2_max=24.0, trials=100)
                       _times(1, trials, 5101, device)[0], facts={"rates": rates})
 
 
+def clean16(device="cpu", n=1 << 26, k=8, dtype=BF16) -> Population:
+    """k fp16 or bf16 candidates of n elements against one reference, every one the narrowed reference plus noise far
+    below the tolerance (sigma 1e-6; atol = rtol = 1e-2): a large, clean 16-bit population, what the outputs of
+    half-precision kernels that are simply right look like."""
+    atol, rtol = 1e-2, 1e-2
+    g = _gen(device, 6000)
+    ref32 = torch.randn(n, generator=g, device=device, dtype=torch.float32)
+    ref = ref32.to(TORCH_DTYPE[dtype])
+    tensors = []
+    for i in range(k):
+        noise = torch.randn(n, generator=g, device=device, dtype=torch.float32)
+        tensors.append(Tensor(noise.mul_(1e-6).add_(ref32).to(TORCH_DTYPE[dtype]), 0, i, dtype))
+    return Population("clean16", [ref], tensors, k, atol, rtol,
+                      _times(k, 100, 6100, device), _times(1, 100, 6101, device)[0])
+
+
 def special_values(dtype=F32, device="cpu") -> Population:
     """Every pair from a set of special values (signed zeros, subnormals, ones and their
     neighbours, the largest finite value, infinities, NaN) as (candidate, reference)."""
