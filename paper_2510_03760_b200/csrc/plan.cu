@@ -57,7 +57,8 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
     // Up to kMaxK.  An item (set, tile) is the unit of the cut below, so a CTA's share is only even to
     // within one item; when every CTA gets work but only a few items (a mid-sized population of many
     // tensors per reference), smaller sets give more, lighter items at the price of reading the
-    // reference once more per extra set (from L2, mostly).
+    // reference once more per extra set (from L2, mostly).  The same holds with more reason when
+    // there are fewer items than CTAs.
     uint32_t cap = kMaxK;
     {
         std::unordered_map<Key, uint32_t, KeyHash> members_of;
@@ -73,8 +74,13 @@ int build_plan(const void* const* cand_ptrs, const void* ref_ptr, const evo_desc
                 items += static_cast<unsigned __int128>((kv.first.n + kTileElems - 1) / kTileElems) * ((kv.second + c - 1) / c);
             return items;
         };
-        if (items_with(kMaxK) >= max_ctas)
+        if (items_with(kMaxK) >= max_ctas) {
             while (cap > 4 && items_with(cap) < static_cast<unsigned __int128>(6) * max_ctas) cap /= 2;
+        } else {
+            // Fewer items than CTAs (a small population): a CTA's time is its start-up plus one member after the
+            // other, so the members are spread over as many CTAs as there are, down to one member per set.
+            while (cap > 1 && items_with(cap) < max_ctas) cap /= 2;
+        }
     }
 
     // ---- sets: tensors with the same (reference, n, dtype), at most `cap` each ----

@@ -95,21 +95,29 @@ def test_few_items_per_cta_split_a_large_set_for_balance(lib):
     tiles = tiles_of(n, F32, int(summ["tile_elems"]))
     w = coverage(summ, ranges, [tiles] * 4)
     assert max(w) <= 1.12 * (sum(w) / len(w))          # shares within one item (5 tiles) of a mean of 46
-    # fewer tiles than CTAs: nothing to balance, one set
+    # fewer items than CTAs (a small population): the members are spread over sets of 2 until there are items for
+    # every CTA - 100 tiles x 8 sets = 800 items for 444 CTAs (sets of 4 would have given 400)
     descs["n"] = 100 * 4096
     st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
-    assert st == 0 and summ["n_sets"] == 1 and summ["n_ctas"] == 100
+    assert st == 0 and summ["n_sets"] == 8 and set_k.tolist() == [2] * 8 and summ["n_ctas"] == 444
+    # a single tile per tensor: every member its own set, sixteen CTAs
+    descs["n"] = 4096
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
+    assert st == 0 and summ["n_sets"] == 16 and set_k.tolist() == [1] * 16 and summ["n_ctas"] == 16
 
 
 def test_more_members_than_a_set_holds(lib):
     descs = np.zeros(100, DESC)
     descs["n"], descs["ref"], descs["dtype"] = 50000, 0x7000_0000_0000, BF16
     cands = 0x1000_0000_0000 + np.arange(100, dtype=np.uint64) * 100096
-    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 64)
-    assert st == 0 and set_k.tolist() == [32, 32, 32, 4]
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 8)
+    assert st == 0 and set_k.tolist() == [32, 32, 32, 4]                  # 52 items for 8 CTAs: as large as sets get
     assert set_of.tolist() == [i // 32 for i in range(100)]
     tiles = tiles_of(50000, BF16, int(summ["tile_elems"]))
     coverage(summ, ranges, [tiles] * 4)
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 64)       # fewer items than CTAs: sets of 16
+    assert st == 0 and set_k.tolist() == [16] * 6 + [4] and set_of.tolist() == [i // 16 for i in range(100)]
+    coverage(summ, ranges, [tiles] * 7)
 
 
 def test_ragged_mixed_population(lib):
@@ -161,10 +169,17 @@ def test_heavy_items_with_few_tiles_leave_no_idle_cta(lib):
     descs["n"], descs["dtype"] = 10000, F16
     descs["ref"][:40], descs["ref"][40:] = 0x7000_0000_0000, 0x7100_0000_0000
     cands = 0x1000_0000_0000 + np.arange(80, dtype=np.uint64) * 65536
-    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 2)
     assert st == 0 and set_k.tolist() == [32, 8, 32, 8] and summ["total_tiles"] == 12
-    assert all(r["set_begin"] <= r["set_end"] for r in ranges) and 0 < summ["n_ctas"] <= 12
+    assert all(r["set_begin"] <= r["set_end"] for r in ranges) and 0 < summ["n_ctas"] <= 2
     coverage(summ, ranges, [3, 3, 3, 3])
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 11)       # boundaries inside heavy items: no empty run
+    assert st == 0 and all(r["set_begin"] <= r["set_end"] for r in ranges) and 0 < summ["n_ctas"] <= 11
+    coverage(summ, ranges, [3] * int(summ["n_sets"]))
+    # with CTAs to spare the same tensors are spread out: one member per set, 240 light items
+    st, summ, ranges, set_of, set_k = inspect(lib, cands, descs, 444)
+    assert st == 0 and set_k.tolist() == [1] * 80 and summ["total_tiles"] == 240 and summ["n_ctas"] == 240
+    coverage(summ, ranges, [3] * 80)
 
 
 def test_empty_and_zero_length(lib):
