@@ -370,6 +370,30 @@ def measure_config(evo, ctx, name, device, peak, reps):
         "kernel": "validate_pass1 (CUDA events around the launch, median)",
         "call": "evo_validate, calls back to back (CUDA events around the loop)",
     }
+    if fits_l2:
+        # Launch-bound populations: the repeated call only launches kernels (the plan is reused), so check + fitness
+        # can be captured once and replayed as a CUDA graph.
+        side = torch.cuda.Stream(device)
+        with torch.cuda.stream(side):
+            for i in range(3):
+                validate(0)
+                evo.evo_fitness(pop.times, pop.base_times, gpass, out=fits, ctx=ctx)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            validate(0)
+            evo.evo_fitness(pop.times, pop.base_times, gpass, out=fits, ctx=ctx)
+        graph.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        out["graph_replay_ms"] = a.elapsed_time(b) / reps
+        out["graph"] = "evo_validate + evo_fitness captured once in a CUDA graph, replays back to back"
+        del graph
     if name == "config5":
         # load balance as measured: every CTA's own begin and end clock in one extra, untimed call
         ctx.cta_timing(True)

@@ -157,7 +157,9 @@ typedef struct {
  * A call whose pointer and descriptor arrays, reference, dtype, groups and stream equal those of
  * the call before it on the same context (an evaluation loop that reuses its buffers for every
  * test case) reuses that call's schedule, which is still in device memory, and only launches the
- * kernels; the tensors are read again, the tolerances may differ.  Schedules of up to 32 KiB
+ * kernels; the tensors are read again, the tolerances may differ.  Such a repeated call makes no
+ * copy, no allocation and no host wait, so after one ordinary call on the stream it can be
+ * captured in a CUDA graph (together with evo_fitness) and replayed.  Schedules of up to 32 KiB
  * (a few hundred tensors) reach the device as kernel arguments, larger ones by a copy from a
  * pinned block of the context.
  * Errors: EVO_ERR_ARG, EVO_ERR_DTYPE, EVO_ERR_ALIGN, EVO_ERR_WORKSPACE, EVO_ERR_CUDA.

@@ -146,3 +146,39 @@ def test_per_cta_clocks_cover_every_cta_and_lie_inside_the_call(evo):
     ctx.cta_timing(False)
     evo.evo_validate(cands, refs, pop.atol, pop.rtol, groups=groups, n_group=pop.n_group, ctx=ctx)
     assert len(ctx.read_cta_times()) == 0
+
+
+def test_a_repeated_call_can_be_captured_in_a_cuda_graph_and_replayed(evo):
+    """After one ordinary call on the stream, the same call only launches kernels (its plan is in device memory), so
+    check and fitness can be captured once and replayed; each replay reads the tensors as they are then."""
+    import oracle
+    ctx = evo.Context(0)
+    pop = workloads.config2("cpu", n=30000, k=5, trials=7)
+    cands, refs, groups = _dev(pop)
+    prep = evo.Prepared(cands, refs, groups, pop.n_group)
+    times, base = pop.times.cuda(), pop.base_times.cuda()
+    res = torch.empty((len(cands), 40), dtype=torch.uint8, device="cuda")
+    gp = torch.empty(pop.n_group, dtype=torch.int32, device="cuda")
+    fit = torch.empty((pop.n_group, 16), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        evo.evo_validate(prep, None, pop.atol, pop.rtol, results=res, group_pass=gp, ctx=ctx)
+        evo.evo_fitness(times, base, gp, out=fit, ctx=ctx)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    before = ctx.launches
+    with torch.cuda.graph(graph, stream=side):
+        evo.evo_validate(prep, None, pop.atol, pop.rtol, results=res, group_pass=gp, ctx=ctx)
+        evo.evo_fitness(times, base, gp, out=fit, ctx=ctx)
+    assert ctx.launches - before == 3                       # first pass, second pass with the verdicts, fitness: no plan store
+    for rnd in range(3):
+        if rnd:
+            cands[rnd].mul_(1.5)                             # in place, between replays
+            pop.tensors[rnd].cand = pop.tensors[rnd].cand * 1.5
+        res.fill_(0xAB)
+        graph.replay()
+        torch.cuda.synchronize()
+        want, verdict = oracle_population(pop)
+        assert_results_equal(evo.results_to_numpy(res), want, "replay %d" % rnd)
+        assert np.array_equal(gp.cpu().numpy().view(np.uint32), verdict)
+        assert evo.fits_to_numpy(fit).tobytes() == oracle.fitness(pop.times.numpy(), pop.base_times.numpy(), verdict).tobytes()
